@@ -1,0 +1,179 @@
+/*
+ * pcomoe.h - C ABI of the path-composed MoE FFN layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer (PCoMoE, Sec. 4): every SwiGLU expert e is split into an expansion-side
+ * operator U_e(h) = SiLU(W_gate h) (.) (W_up h) and a projection-side operator
+ * D_e(a) = W_down a.  A path (i,j) composes source i with target j, P_ij(h) = D_j(U_i(h)).
+ * Per token the router scores the paths allowed by a layer-wise compatibility mask,
+ * keeps the K best, and the layer returns  y = sum_{(i,j) in Pi(h)} beta_ij P_ij(h).
+ * A U_i(h) needed by several of a token's paths is computed once and reused.
+ *
+ * Conventions
+ *   - Row-major arrays.  Weights are [out_features, in_features]:
+ *       W_gate, W_up [n, F, H];  W_down [n, H, F];  shared expert [F_sh, H], [F_sh, H], [H, F_sh].
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; h_* are HOST pointers.
+ *     The three hot calls allocate and free nothing.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Hot calls only enqueue work on it and return; they never synchronise.
+ *   - Host-detectable problems are returned at once as a pcomoe_status and nothing is
+ *     enqueued.  Problems only the device can see (an index out of range, a wait that ran
+ *     out) are written to a status word in the workspace: read it with pcomoe_device_status.
+ *     Nothing throws, aborts or traps.
+ *   - int32 indices (T*K < 2^31).  T = 0 is a valid no-op.  Empty groups are legal.
+ */
+#ifndef PCOMOE_H_
+#define PCOMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PCOMOE_OK = 0,
+  PCOMOE_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, bad enum, mask without its diagonal */
+  PCOMOE_ERR_SHAPE = 2,       /* T larger than the workspace was sized for, K > n, ...            */
+  PCOMOE_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small                       */
+  PCOMOE_ERR_UNSUPPORTED = 4, /* a size or dtype combination no kernel covers                     */
+  PCOMOE_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                              */
+  PCOMOE_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out                   */
+  PCOMOE_ERR_INDEX = 7        /* device: an expert / row index was out of range                   */
+} pcomoe_status;
+
+typedef enum { PCOMOE_BF16 = 0, PCOMOE_FP32 = 1 } pcomoe_dtype;
+
+/* Which kernels pcomoe_ffn_forward uses. */
+typedef enum {
+  PCOMOE_FFN_AUTO = 0,   /* tensor-core path when dtype and sizes allow, else the SIMT path */
+  PCOMOE_FFN_SIMT = 1,   /* plain-FMA kernels (any size, bf16 or fp32 storage)               */
+  PCOMOE_FFN_TCGEN05 = 2 /* tcgen05 / TMEM / TMA kernels; PCOMOE_ERR_UNSUPPORTED if not bf16
+                            or if H % 256 != 0 or F % 128 != 0                               */
+} pcomoe_ffn_impl;
+
+/* Plain data; set struct_size = sizeof(pcomoe_config). */
+typedef struct {
+  int32_t struct_size;
+  int32_t n_experts;    /* n                                                                  */
+  int32_t top_k;        /* K paths per token, 1 <= K <= min(n, 32)                            */
+  int32_t hidden;       /* H                                                                  */
+  int32_t ffn;          /* F, per-expert intermediate width                                   */
+  int32_t shared_ffn;   /* F_sh, width of the always-on shared expert; 0 = none               */
+  int32_t in_dtype;     /* pcomoe_dtype of h and of every weight                              */
+  int32_t out_dtype;    /* pcomoe_dtype of y; only PCOMOE_FP32 is implemented                 */
+  float lambda;         /* scale of the target-side prior in the path score (Sec. 4.2)        */
+  int32_t norm_topk;    /* 1: beta = softmax over the K selected scores;
+                           0: softmax over the whole active set, gathered at the K selected   */
+  float routed_scale;   /* every beta is multiplied by this (1.0 = plain)                     */
+  int32_t dedup;        /* 1: one stage-1 row per unique (token, source)  (Sec. 4.3 reuse);
+                           0: one stage-1 row per path                                        */
+  int32_t ffn_impl;     /* pcomoe_ffn_impl                                                    */
+} pcomoe_config;
+
+typedef struct pcomoe_layer pcomoe_layer; /* opaque; owns the small device table of active paths */
+
+/*
+ * Layer set-up (offline, once per layer).  Builds the active set A = {(i,j) | m_ij = 1}
+ * (Sec. 4.3, "Compositional Path Routing": path indices are materialised offline) as a compact
+ * table sorted by flat id i*n+j, and copies it to the current device (the one call here that
+ * allocates device memory; pcomoe_layer_destroy frees it).
+ *   h_mask [n*n] uint8, row i = source, column j = target; every m_ii must be 1 (Sec. 4.2).
+ *   h_bias [n*n] fp32 compatibility bias B; entries where the mask is 0 are never read.
+ * Errors: INVALID_ARG (NULL, sizes <= 0, diagonal entry off), SHAPE (K > n or K > 32),
+ * UNSUPPORTED (n > 256, H or F not a multiple of 8, F_sh not a multiple of 8), CUDA.
+ */
+pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mask,
+                                  const float *h_bias, pcomoe_layer **out);
+pcomoe_status pcomoe_layer_destroy(pcomoe_layer *layer);
+
+/* Number of active paths |A| of the layer; copies up to `cap` table entries to host arrays
+ * (any of them may be NULL).  For checking the table against the mask. */
+pcomoe_status pcomoe_layer_active_set(const pcomoe_layer *layer, int32_t cap, int32_t *h_src,
+                                      int32_t *h_tgt, float *h_bias, int32_t *count);
+
+/* Bytes of device workspace pcomoe_build_path_groups and pcomoe_ffn_forward need for up to
+ * max_tokens tokens.  The workspace must be 256-byte aligned. */
+pcomoe_status pcomoe_workspace_bytes(const pcomoe_layer *layer, int32_t max_tokens, size_t *bytes);
+
+/*
+ * Path routing (Sec. 4.2 score equation, Sec. 4.3 TopK equation).  For every token t and every
+ * active path a = (i,j):
+ *     s_a = (z[t,i] + b_ij) + lambda * u[t,j]        three fp32 operations, each rounded, no FMA
+ * Pi(t) = the K paths largest under (score descending, flat id i*n+j ascending); beta as
+ * cfg.norm_topk says, times cfg.routed_scale.
+ *   d_logits     [T,n] fp32  base routing signal z (pre-softmax router logits), finite values
+ *   d_tgt_logits [T,n] fp32  projection-side prior u, or NULL to use d_logits
+ *   d_path_src, d_path_tgt [T,K] int32 and d_path_w [T,K] fp32: outputs in rank order.
+ * One warp per token; no workspace.  Errors: INVALID_ARG, SHAPE (T < 0), CUDA (launch failure).
+ */
+pcomoe_status pcomoe_route_paths(const pcomoe_layer *layer, int32_t T, const float *d_logits,
+                                 const float *d_tgt_logits, int32_t *d_path_src,
+                                 int32_t *d_path_tgt, float *d_path_w, void *stream);
+
+/* Device arrays filled by pcomoe_build_path_groups; all caller-allocated.
+ *   s1_offsets [n+1]  stage-1 (expansion) rows of source i are [s1_offsets[i], s1_offsets[i+1])
+ *   s1_token   [T*K]  token of each stage-1 row (first R1 = s1_offsets[n] entries are written)
+ *   path_s1row [T,K]  stage-1 row that path (t,k) reads its intermediate from
+ *   s2_offsets [n+1]  stage-2 (projection) rows of target j
+ *   s2_path    [T*K]  flat path id t*K+k of each stage-2 row
+ *   s2_s1row   [T*K]  = path_s1row[s2_path]
+ *   s2_token   [T*K]  = s2_path / K
+ *   s2_w       [T*K]  = path_w[s2_path]
+ *   stats      [8]    R1, P, stage-1 tiles, stage-2 tiles, empty source groups, empty target
+ *                     groups, 0, 0
+ */
+typedef struct {
+  int32_t *s1_offsets, *s1_token, *path_s1row, *s2_offsets, *s2_path, *s2_s1row, *s2_token;
+  float *s2_w;
+  int32_t *stats;
+} pcomoe_groups;
+
+/*
+ * Source grouping with reuse, and target grouping (Sec. 4.3, "Source-Grouped Compute Reuse":
+ * S(h) and T_i(h)).  A stage-1 slot is a unique (token, source) pair (cfg.dedup = 1) or a path
+ * (cfg.dedup = 0).  Orders are canonical, so the result is unique:
+ *   stage-1 rows by (source ascending, token ascending)  [dedup = 0: (source, flat path id)]
+ *   stage-2 rows by (target ascending, flat path id t*K+k ascending).
+ * Histogram, prefix scan and stable scatter; integer work only.  Also leaves in the workspace
+ * the tile schedule and padded gather maps that pcomoe_ffn_forward reads, so the same
+ * d_workspace must be passed to the following pcomoe_ffn_forward.
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.  Device: INDEX if a source/target is outside [0,n).
+ */
+pcomoe_status pcomoe_build_path_groups(const pcomoe_layer *layer, int32_t T,
+                                       const int32_t *d_path_src, const int32_t *d_path_tgt,
+                                       const float *d_path_w, const pcomoe_groups *out,
+                                       void *d_workspace, size_t ws_bytes, void *stream);
+
+/*
+ * Layer forward over the groups (Sec. 4.1 operators U_e, D_e; Sec. 4.3 source-grouped output):
+ *   stage 1  for each source i and each of its rows r:  U[r,:] = SiLU(W_gate^(i) h_t) (.) (W_up^(i) h_t),
+ *            t = s1_token[r]                 (bf16 storage: fp32 accumulate, U kept in bf16)
+ *   stage 2  for each target j and each of its rows q:
+ *            y[s2_token[q],:] += s2_w[q] * W_down^(j) U[s2_s1row[q],:]   (fp32 accumulate and add)
+ *   shared   y[t,:] += Wsh_down (SiLU(Wsh_gate h_t) (.) (Wsh_up h_t))  when F_sh > 0 (weight 1).
+ *   d_h [T,H]; d_w_gate, d_w_up [n,F,H]; d_w_down [n,H,F]; shared weights or NULL (all in in_dtype);
+ *   d_y [T,H] fp32, fully overwritten (zero-filled first, then accumulated with atomic adds, so the
+ *   order of the additions - and the last bits of y - can differ between calls).
+ * `groups` and d_workspace must come from pcomoe_build_path_groups for the same T.
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE, UNSUPPORTED, CUDA.  Device: TIMEOUT, INDEX.
+ */
+pcomoe_status pcomoe_ffn_forward(const pcomoe_layer *layer, int32_t T, const void *d_h,
+                                 const void *d_w_gate, const void *d_w_up, const void *d_w_down,
+                                 const void *d_wsh_gate, const void *d_wsh_up,
+                                 const void *d_wsh_down, const pcomoe_groups *groups, void *d_y,
+                                 void *d_workspace, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, reads the workspace's status word and returns the first error a kernel
+ * recorded (PCOMOE_OK if none); the word is cleared by the next pcomoe_build_path_groups. */
+pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream);
+
+/* Launch counters (kernels and memsets enqueued by this library since load, per process). */
+int64_t pcomoe_launch_count(void);
+
+const char *pcomoe_status_string(pcomoe_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PCOMOE_H_ */

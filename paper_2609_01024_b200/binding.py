@@ -1,0 +1,279 @@
+"""ctypes binding of libpcomoe.so: same names as the C ABI, argument marshalling only.
+
+PyTorch provides device memory and streams; every step of the layer runs in the library's
+kernels.  There is no fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libpcomoe.so")
+
+PCOMOE_OK = 0
+STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_WORKSPACE", 4: "ERR_UNSUPPORTED",
+                5: "ERR_CUDA", 6: "ERR_TIMEOUT", 7: "ERR_INDEX"}
+PCOMOE_BF16, PCOMOE_FP32 = 0, 1
+PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05 = 0, 1, 2
+
+EXPORTS = ["pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
+           "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_ffn_forward", "pcomoe_device_status",
+           "pcomoe_launch_count", "pcomoe_status_string"]
+
+
+class PcomoeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        super().__init__(f"{where}: PCOMOE_{STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+class pcomoe_config(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_int32), ("n_experts", ctypes.c_int32), ("top_k", ctypes.c_int32),
+                ("hidden", ctypes.c_int32), ("ffn", ctypes.c_int32), ("shared_ffn", ctypes.c_int32),
+                ("in_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32), ("lambda_", ctypes.c_float),
+                ("norm_topk", ctypes.c_int32), ("routed_scale", ctypes.c_float), ("dedup", ctypes.c_int32),
+                ("ffn_impl", ctypes.c_int32)]
+
+
+class pcomoe_groups(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_void_p) for k in ("s1_offsets", "s1_token", "path_s1row", "s2_offsets", "s2_path",
+                                                "s2_s1row", "s2_token", "s2_w", "stats")]
+
+
+_lib = None
+
+
+def load_library(path: str | None = None):
+    """Loads libpcomoe.so; raises if it has not been built (no CPU or eager fallback exists)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(f"{p} not found: build it with `python -m paper_2609_01024_b200.build`")
+    lib = ctypes.CDLL(p)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    lib.pcomoe_layer_create.argtypes = [ctypes.POINTER(pcomoe_config), vp, vp, ctypes.POINTER(vp)]
+    lib.pcomoe_layer_destroy.argtypes = [vp]
+    lib.pcomoe_layer_active_set.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(i32)]
+    lib.pcomoe_workspace_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
+    lib.pcomoe_route_paths.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.pcomoe_build_path_groups.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, sz, vp]
+    lib.pcomoe_ffn_forward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
+    lib.pcomoe_device_status.argtypes = [vp, vp]
+    lib.pcomoe_launch_count.restype = ctypes.c_int64
+    lib.pcomoe_status_string.restype = ctypes.c_char_p
+    lib.pcomoe_status_string.argtypes = [i32]
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _check(status: int, where: str):
+    if status != PCOMOE_OK:
+        raise PcomoeError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def pcomoe_launch_count() -> int:
+    return int(load_library().pcomoe_launch_count())
+
+
+def pcomoe_layer_create(*, n_experts, top_k, hidden, ffn, mask, bias, shared_ffn=0, in_dtype=PCOMOE_BF16,
+                        out_dtype=PCOMOE_FP32, lam=0.5, norm_topk=1, routed_scale=1.0, dedup=1,
+                        ffn_impl=PCOMOE_FFN_AUTO):
+    lib = load_library()
+    cfg = pcomoe_config(ctypes.sizeof(pcomoe_config), n_experts, top_k, hidden, ffn, shared_ffn, in_dtype,
+                        out_dtype, lam, norm_topk, routed_scale, dedup, ffn_impl)
+    m = np.ascontiguousarray(mask, dtype=np.uint8)
+    b = np.ascontiguousarray(bias, dtype=np.float32)
+    assert m.size == n_experts * n_experts and b.size == n_experts * n_experts
+    out = ctypes.c_void_p()
+    _check(lib.pcomoe_layer_create(ctypes.byref(cfg), m.ctypes.data_as(ctypes.c_void_p),
+                                   b.ctypes.data_as(ctypes.c_void_p), ctypes.byref(out)), "pcomoe_layer_create")
+    return out
+
+
+def pcomoe_layer_destroy(layer):
+    _check(load_library().pcomoe_layer_destroy(layer), "pcomoe_layer_destroy")
+
+
+def pcomoe_layer_active_set(layer, n_experts):
+    cap = n_experts * n_experts
+    src = np.zeros(cap, np.int32); tgt = np.zeros(cap, np.int32); b = np.zeros(cap, np.float32)
+    cnt = ctypes.c_int32(0)
+    _check(load_library().pcomoe_layer_active_set(layer, cap, src.ctypes.data_as(ctypes.c_void_p),
+                                                  tgt.ctypes.data_as(ctypes.c_void_p),
+                                                  b.ctypes.data_as(ctypes.c_void_p), ctypes.byref(cnt)),
+           "pcomoe_layer_active_set")
+    return src[:cnt.value].copy(), tgt[:cnt.value].copy(), b[:cnt.value].copy()
+
+
+def pcomoe_workspace_bytes(layer, max_tokens: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().pcomoe_workspace_bytes(layer, max_tokens, ctypes.byref(n)), "pcomoe_workspace_bytes")
+    return int(n.value)
+
+
+def pcomoe_route_paths(layer, T, logits, tgt_logits, path_src, path_tgt, path_w):
+    _check(load_library().pcomoe_route_paths(layer, T, _ptr(logits), _ptr(tgt_logits), _ptr(path_src),
+                                             _ptr(path_tgt), _ptr(path_w), _stream()), "pcomoe_route_paths")
+
+
+class Groups:
+    """Device arrays of one pcomoe_build_path_groups call (torch tensors own the memory)."""
+    FIELDS = ("s1_offsets", "s1_token", "path_s1row", "s2_offsets", "s2_path", "s2_s1row", "s2_token", "s2_w", "stats")
+
+    def __init__(self, T: int, K: int, n: int, device):
+        P = max(T * K, 1)
+        i32 = dict(dtype=torch.int32, device=device)
+        self.s1_offsets = torch.zeros(n + 1, **i32)
+        self.s1_token = torch.zeros(P, **i32)
+        self.path_s1row = torch.zeros(max(T, 1), K, **i32)
+        self.s2_offsets = torch.zeros(n + 1, **i32)
+        self.s2_path = torch.zeros(P, **i32)
+        self.s2_s1row = torch.zeros(P, **i32)
+        self.s2_token = torch.zeros(P, **i32)
+        self.s2_w = torch.zeros(P, dtype=torch.float32, device=device)
+        self.stats = torch.zeros(8, **i32)
+        self.T, self.K, self.n = T, K, n
+        self.c = pcomoe_groups(*[ctypes.c_void_p(getattr(self, f).data_ptr()) for f in self.FIELDS])
+
+    def to_host(self):
+        P = self.T * self.K
+        out = {f: getattr(self, f).cpu().numpy() for f in self.FIELDS}
+        out["R1"] = int(out["stats"][0])
+        out["s1_token"] = out["s1_token"][:out["R1"]]
+        out["path_s1row"] = out["path_s1row"][:self.T]
+        for f in ("s2_path", "s2_s1row", "s2_token", "s2_w"):
+            out[f] = out[f][:P]
+        return out
+
+
+def pcomoe_build_path_groups(layer, T, path_src, path_tgt, path_w, groups: Groups, workspace):
+    _check(load_library().pcomoe_build_path_groups(layer, T, _ptr(path_src), _ptr(path_tgt), _ptr(path_w),
+                                                   ctypes.byref(groups.c), _ptr(workspace),
+                                                   workspace.numel() * workspace.element_size(), _stream()),
+           "pcomoe_build_path_groups")
+
+
+def pcomoe_ffn_forward(layer, T, h, w_gate, w_up, w_down, wsh_gate, wsh_up, wsh_down, groups: Groups, y, workspace):
+    _check(load_library().pcomoe_ffn_forward(layer, T, _ptr(h), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                                             _ptr(wsh_gate), _ptr(wsh_up), _ptr(wsh_down), ctypes.byref(groups.c),
+                                             _ptr(y), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                             _stream()), "pcomoe_ffn_forward")
+
+
+def pcomoe_device_status(workspace) -> int:
+    return int(load_library().pcomoe_device_status(_ptr(workspace), _stream()))
+
+
+class PathMoELayer:
+    """Owns the device buffers of one layer and chains the three hot calls.  Marshalling only."""
+
+    def __init__(self, *, n_experts, top_k, hidden, ffn, mask, bias, w_gate, w_up, w_down, shared=None,
+                 max_tokens, in_dtype=PCOMOE_BF16, lam=0.5, norm_topk=1, routed_scale=1.0, dedup=1,
+                 ffn_impl=PCOMOE_FFN_AUTO, device="cuda:0"):
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.n, self.K, self.H, self.F = n_experts, top_k, hidden, ffn
+        self.F_sh = 0 if shared is None or shared[0] is None else int(shared[0].shape[0])
+        self.layer = pcomoe_layer_create(n_experts=n_experts, top_k=top_k, hidden=hidden, ffn=ffn, mask=mask,
+                                         bias=bias, shared_ffn=self.F_sh, in_dtype=in_dtype, lam=lam,
+                                         norm_topk=norm_topk, routed_scale=routed_scale, dedup=dedup,
+                                         ffn_impl=ffn_impl)
+        self.w_gate, self.w_up, self.w_down = w_gate, w_up, w_down
+        self.shared = shared if self.F_sh else (None, None, None)
+        self.max_tokens = max_tokens
+        self.workspace = torch.empty(pcomoe_workspace_bytes(self.layer, max_tokens), dtype=torch.uint8,
+                                     device=self.device)
+        assert self.workspace.data_ptr() % 256 == 0
+        T = max(max_tokens, 1)
+        self.path_src = torch.zeros(T, top_k, dtype=torch.int32, device=self.device)
+        self.path_tgt = torch.zeros(T, top_k, dtype=torch.int32, device=self.device)
+        self.path_w = torch.zeros(T, top_k, dtype=torch.float32, device=self.device)
+        self.groups = Groups(max_tokens, top_k, n_experts, self.device)
+        self.y = torch.zeros(T, hidden, dtype=torch.float32, device=self.device)
+        self.in_torch_dtype = torch.bfloat16 if in_dtype == PCOMOE_BF16 else torch.float32
+        self._pin_logits = self._pin_h = self._pin_y = None
+        self._d_logits = self._d_h = None
+
+    def close(self):
+        if self.layer is not None:
+            pcomoe_layer_destroy(self.layer)
+            self.layer = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def route(self, logits, tgt_logits=None):
+        T = logits.shape[0]
+        pcomoe_route_paths(self.layer, T, logits, tgt_logits, self.path_src, self.path_tgt, self.path_w)
+
+    def build_groups(self, T):
+        self.groups.T = T
+        pcomoe_build_path_groups(self.layer, T, self.path_src, self.path_tgt, self.path_w, self.groups, self.workspace)
+
+    def ffn(self, h):
+        T = h.shape[0]
+        pcomoe_ffn_forward(self.layer, T, h, self.w_gate, self.w_up, self.w_down, *self.shared, self.groups,
+                           self.y, self.workspace)
+
+    def forward(self, logits, h, tgt_logits=None):
+        """The whole hot path on device tensors: route -> group -> stage 1 -> stage 2.  Returns y [T,H] fp32."""
+        T = h.shape[0]
+        assert T <= self.max_tokens
+        self.route(logits, tgt_logits)
+        self.build_groups(T)
+        self.ffn(h)
+        return self.y[:T]
+
+    def forward_host(self, logits_np: np.ndarray, h_np: np.ndarray) -> np.ndarray:
+        """End to end from host buffers: pinned H2D copies of logits and hidden states, the hot path,
+        and a D2H copy of y.  `h_np` is fp32, or uint16 bf16 bit patterns for a bf16 layer."""
+        T = h_np.shape[0]
+        if self._pin_logits is None or self._pin_logits.shape[0] < T:
+            cap = max(T, self.max_tokens)
+            self._pin_logits = torch.empty(cap, self.n, dtype=torch.float32).pin_memory()
+            hdt = torch.float32 if h_np.dtype == np.float32 else torch.int16
+            self._pin_h = torch.empty(cap, self.H, dtype=hdt).pin_memory()
+            self._pin_y = torch.empty(cap, self.H, dtype=torch.float32).pin_memory()
+            self._d_logits = torch.empty(cap, self.n, dtype=torch.float32, device=self.device)
+            self._d_h = torch.empty(cap, self.H, dtype=hdt, device=self.device)
+        self._pin_logits[:T].numpy()[...] = logits_np
+        self._pin_h[:T].numpy()[...] = h_np.view(np.int16) if h_np.dtype == np.uint16 else h_np
+        self._d_logits[:T].copy_(self._pin_logits[:T], non_blocking=True)
+        self._d_h[:T].copy_(self._pin_h[:T], non_blocking=True)
+        dh = self._d_h[:T]
+        if dh.dtype == torch.int16:
+            dh = dh.view(torch.bfloat16)
+        y = self.forward(self._d_logits[:T], dh)
+        self._pin_y[:T].copy_(y, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return self._pin_y[:T].numpy()
+
+    def device_status(self) -> int:
+        return pcomoe_device_status(self.workspace)
+
+
+def to_device(arr: np.ndarray | None, device="cuda:0"):
+    """numpy -> device tensor; uint16 arrays are bf16 bit patterns."""
+    if arr is None:
+        return None
+    if arr.dtype == np.uint16:
+        return torch.from_numpy(arr.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(arr).to(device)

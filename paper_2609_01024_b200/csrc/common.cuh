@@ -1,0 +1,95 @@
+// Internal declarations shared by the translation units of libpcomoe.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pcomoe.h"
+
+namespace pcomoe {
+
+constexpr int kTileM = 128;        // rows of one GEMM tile (one TMEM lane per row)
+constexpr int kMaxExperts = 256;
+constexpr int kMaxTopK = 32;
+
+// One entry of the active-path table (sorted by flat id src*n+tgt).
+struct __align__(8) ActiveEntry {
+  uint16_t src;
+  uint16_t tgt;
+  float bias;
+};
+
+// Device-side header at the start of the workspace.
+struct DevPlan {
+  int32_t status;      // first device-detected error (pcomoe_status), 0 if none
+  int32_t R1;          // stage-1 rows
+  int32_t P;           // stage-2 rows (= T*K)
+  int32_t mt1;         // 128-row tiles of stage 1 (sum over sources of ceil(rows/128))
+  int32_t mt2;         // 128-row tiles of stage 2
+  int32_t empty1;      // sources without rows
+  int32_t empty2;      // targets without rows
+  int32_t T;           // tokens of the last pcomoe_build_path_groups
+};
+
+// Byte offsets of the workspace sections (all multiples of 256).
+struct WsLayout {
+  size_t plan;         // DevPlan
+  size_t tile_base1;   // int32 [n+1]   prefix of stage-1 m-tiles per source
+  size_t tile_base2;   // int32 [n+1]   prefix of stage-2 m-tiles per target
+  size_t blk_cnt;      // int32 [NB][2][n] per-block histograms, turned into offsets by the scan
+  size_t a1_idx;       // int32 [mt_max*128] token of every padded stage-1 row
+  size_t a2_idx;       // int32 [mt_max*128] padded U row of every padded stage-2 row
+  size_t u;            // in_dtype [mt_max*128, F]   intermediates, groups padded to 128 rows
+  size_t u_sh;         // in_dtype [Tpad, F_sh]      shared-expert intermediates
+  size_t a_perm1;      // bf16 [mt_max*128, H]  (only when the gather-free fallback is enabled)
+  size_t a_perm2;      // bf16 [mt_max*128, F]
+  size_t total;
+  int32_t nb_max;      // blocks of the grouping kernels at max_tokens
+  int32_t mt_max;      // upper bound of m-tiles per stage
+  int32_t t_pad;       // max_tokens rounded up to 128
+};
+
+}  // namespace pcomoe
+
+struct pcomoe_layer {
+  pcomoe_config cfg;
+  int32_t n_active;                 // |A|
+  pcomoe::ActiveEntry *d_table;     // device copy of the active-path table
+  pcomoe::ActiveEntry *h_table;     // host copy
+  int device;
+  int sm_count;
+  int group_chunk;                  // tokens per block of the grouping kernels
+  int use_gather4;                  // A operand of the GEMMs fetched by TMA gather4 (else pre-permuted)
+  int tc_ok;                        // sizes and dtype allow the tcgen05 path
+};
+
+namespace pcomoe {
+
+WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens);
+void count_launch(int n = 1);
+
+inline size_t dtype_size(int dt) { return dt == PCOMOE_BF16 ? 2 : 4; }
+
+#define PCOMOE_CUDA_TRY(expr)                          \
+  do {                                                 \
+    cudaError_t _e = (expr);                           \
+    if (_e != cudaSuccess) return PCOMOE_ERR_CUDA;     \
+  } while (0)
+
+// launchers implemented in the kernel translation units
+pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, const float *u,
+                           int32_t *src, int32_t *tgt, float *w, cudaStream_t st);
+pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src, const int32_t *tgt,
+                            const float *w, const pcomoe_groups *g, char *ws, const WsLayout &lay,
+                            cudaStream_t st);
+pcomoe_status launch_ffn_simt(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
+                              const void *wu, const void *wd, const void *sg, const void *su,
+                              const void *sd, const pcomoe_groups *g, float *y, char *ws,
+                              const WsLayout &lay, cudaStream_t st);
+pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
+                            const void *wu, const void *wd, const void *sg, const void *su,
+                            const void *sd, const pcomoe_groups *g, float *y, char *ws,
+                            const WsLayout &lay, cudaStream_t st);
+
+}  // namespace pcomoe

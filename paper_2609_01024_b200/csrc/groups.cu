@@ -1,0 +1,251 @@
+// K2: source grouping with reuse and target grouping (Sec. 4.3, "Source-Grouped Compute Reuse").
+//
+// A stable counting sort in three launches, bit-exact and free of inter-block waiting:
+//   count    each block histograms the sources (first occurrences only when reuse is on) and the
+//            targets of its contiguous chunk of tokens;
+//   scan     one block turns the per-block histograms into per-block offsets, the per-expert
+//            offsets, and the 128-row tile schedule of the two GEMM stages;
+//   scatter  each block ranks its own paths with a bit matrix [expert][flat id in chunk]
+//            (rank = set bits below mine) and writes every output at its final position.
+// Orders are canonical: stage-1 rows by (source, token) - or (source, flat path id) without
+// reuse - and stage-2 rows by (target, flat path id).
+#include "common.cuh"
+
+namespace pcomoe {
+
+struct GroupParams {
+  const int32_t *src;   // [T,K]
+  const int32_t *tgt;   // [T,K]
+  const float *w;       // [T,K]
+  pcomoe_groups g;
+  DevPlan *plan;
+  int32_t *tile_base1, *tile_base2;   // [n+1]
+  int32_t *blk_cnt;                   // [NB][2][n]
+  int32_t *a1_idx, *a2_idx;
+  int32_t T, n, K, dedup, chunk, nb;
+};
+
+__device__ __forceinline__ void flag_error(DevPlan *plan, int code) { atomicCAS(&plan->status, 0, code); }
+
+// Loads the block's chunk of path sources / targets into shared memory; returns tokens in chunk.
+__device__ __forceinline__ int stage_chunk(const GroupParams &p, int32_t *ssrc, int32_t *stgt) {
+  const int t0 = blockIdx.x * p.chunk;
+  const int nt = min(p.chunk, p.T - t0);
+  const size_t base = (size_t)t0 * p.K;
+  for (int x = threadIdx.x; x < nt * p.K; x += blockDim.x) {
+    int s = p.src[base + x], t = p.tgt[base + x];
+    if ((unsigned)s >= (unsigned)p.n || (unsigned)t >= (unsigned)p.n) {
+      flag_error(p.plan, PCOMOE_ERR_INDEX);
+      s = -1;  // the path is skipped everywhere
+      t = -1;
+    }
+    ssrc[x] = s;
+    stgt[x] = t;
+  }
+  return nt;
+}
+
+__device__ __forceinline__ int first_occurrence(const int32_t *row, int k, int dedup) {
+  if (!dedup) return k;
+  for (int k2 = 0; k2 < k; ++k2)
+    if (row[k2] == row[k]) return k2;
+  return k;
+}
+
+__global__ void group_count_kernel(const GroupParams p) {
+  extern __shared__ int32_t sm[];
+  int32_t *ssrc = sm, *stgt = sm + p.chunk * p.K;
+  int32_t *h1 = stgt + p.chunk * p.K, *h2 = h1 + p.n;
+  for (int e = threadIdx.x; e < 2 * p.n; e += blockDim.x) h1[e] = 0;
+  const int nt = stage_chunk(p, ssrc, stgt);
+  __syncthreads();
+  if ((int)threadIdx.x < nt) {
+    const int32_t *rs = ssrc + threadIdx.x * p.K, *rt = stgt + threadIdx.x * p.K;
+    for (int k = 0; k < p.K; ++k) {
+      if (rs[k] < 0) continue;
+      if (first_occurrence(rs, k, p.dedup) == k) atomicAdd(&h1[rs[k]], 1);
+      atomicAdd(&h2[rt[k]], 1);
+    }
+  }
+  __syncthreads();
+  int32_t *out = p.blk_cnt + (size_t)blockIdx.x * 2 * p.n;
+  for (int e = threadIdx.x; e < 2 * p.n; e += blockDim.x) out[e] = h1[e];
+}
+
+__device__ __forceinline__ int warp_incl_scan(int v, int lane) {
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, v, off);
+    if (lane >= off) v += o;
+  }
+  return v;
+}
+
+__global__ void __launch_bounds__(1024) group_scan_kernel(const GroupParams p) {
+  __shared__ int32_t tot[2 * kMaxExperts];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+  // (stage, expert) columns: exclusive prefix over the blocks, in place
+  for (int col = warp; col < 2 * p.n; col += warps) {
+    int carry = 0;
+    for (int b0 = 0; b0 < p.nb; b0 += 32) {
+      const int b = b0 + lane;
+      const int v = b < p.nb ? p.blk_cnt[(size_t)b * 2 * p.n + col] : 0;
+      const int incl = warp_incl_scan(v, lane);
+      if (b < p.nb) p.blk_cnt[(size_t)b * 2 * p.n + col] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) tot[col] = carry;
+  }
+  __syncthreads();
+  // warp 0: stage 1, warp 1: stage 2.  Offsets over the experts and the m-tile schedule.
+  if (warp < 2) {
+    const int32_t *cnt = tot + warp * p.n;
+    int32_t *offs = warp == 0 ? p.g.s1_offsets : p.g.s2_offsets;
+    int32_t *tb = warp == 0 ? p.tile_base1 : p.tile_base2;
+    int carry_rows = 0, carry_tiles = 0, empty = 0;
+    for (int e0 = 0; e0 < p.n; e0 += 32) {
+      const int e = e0 + lane;
+      const int c = e < p.n ? cnt[e] : 0;
+      const int tl = (c + kTileM - 1) / kTileM;
+      const int ir = warp_incl_scan(c, lane), it = warp_incl_scan(tl, lane);
+      if (e < p.n) {
+        offs[e] = carry_rows + ir - c;
+        tb[e] = carry_tiles + it - tl;
+      }
+      empty += __popc(__ballot_sync(0xffffffffu, e < p.n && c == 0));
+      carry_rows += __shfl_sync(0xffffffffu, ir, 31);
+      carry_tiles += __shfl_sync(0xffffffffu, it, 31);
+    }
+    if (lane == 0) {
+      offs[p.n] = carry_rows;
+      tb[p.n] = carry_tiles;
+      if (warp == 0) {
+        p.plan->R1 = carry_rows; p.plan->mt1 = carry_tiles; p.plan->empty1 = empty;
+        p.plan->T = p.T;
+        p.g.stats[0] = carry_rows; p.g.stats[2] = carry_tiles; p.g.stats[4] = empty;
+        p.g.stats[6] = 0; p.g.stats[7] = 0;
+      } else {
+        p.plan->P = carry_rows; p.plan->mt2 = carry_tiles; p.plan->empty2 = empty;
+        p.g.stats[1] = carry_rows; p.g.stats[3] = carry_tiles; p.g.stats[5] = empty;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ int bits_below(const uint32_t *row, int idx) {
+  int r = 0;
+  const int word = idx >> 5;
+  for (int w = 0; w < word; ++w) r += __popc(row[w]);
+  return r + __popc(row[word] & ((1u << (idx & 31)) - 1u));
+}
+
+__global__ void group_scatter_kernel(const GroupParams p) {
+  extern __shared__ int32_t sm[];
+  const int CK = p.chunk * p.K;
+  const int W = (CK + 31) >> 5;
+  int32_t *ssrc = sm, *stgt = ssrc + CK, *srow = stgt + CK;
+  int32_t *off1 = srow + CK, *off2 = off1 + p.n, *tb1 = off2 + p.n, *tb2 = tb1 + p.n;
+  int32_t *bo1 = tb2 + p.n, *bo2 = bo1 + p.n;
+  uint32_t *bits1 = reinterpret_cast<uint32_t *>(bo2 + p.n), *bits2 = bits1 + (size_t)p.n * W;
+
+  for (int x = threadIdx.x; x < 2 * p.n * W; x += blockDim.x) bits1[x] = 0u;
+  const int32_t *bo = p.blk_cnt + (size_t)blockIdx.x * 2 * p.n;
+  for (int e = threadIdx.x; e < p.n; e += blockDim.x) {
+    off1[e] = p.g.s1_offsets[e];
+    off2[e] = p.g.s2_offsets[e];
+    tb1[e] = p.tile_base1[e];
+    tb2[e] = p.tile_base2[e];
+    bo1[e] = bo[e];
+    bo2[e] = bo[p.n + e];
+  }
+  const int nt = stage_chunk(p, ssrc, stgt);
+  __syncthreads();
+
+  const int tl = threadIdx.x;
+  const int32_t *rs = ssrc + tl * p.K, *rt = stgt + tl * p.K;
+  if (tl < nt) {
+    for (int k = 0; k < p.K; ++k) {
+      if (rs[k] < 0) continue;
+      const int idx = tl * p.K + k;
+      if (first_occurrence(rs, k, p.dedup) == k) atomicOr(&bits1[(size_t)rs[k] * W + (idx >> 5)], 1u << (idx & 31));
+      atomicOr(&bits2[(size_t)rt[k] * W + (idx >> 5)], 1u << (idx & 31));
+    }
+  }
+  __syncthreads();
+  if (tl >= nt) return;
+
+  const int t = blockIdx.x * p.chunk + tl;
+  int32_t *myrow = srow + tl * p.K;
+  for (int k = 0; k < p.K; ++k) {
+    const int s = rs[k];
+    if (s < 0) continue;
+    const int fk = first_occurrence(rs, k, p.dedup);
+    if (fk == k) {
+      const int idx = tl * p.K + k;
+      const int row = off1[s] + bo1[s] + bits_below(bits1 + (size_t)s * W, idx);
+      myrow[k] = row;
+      p.g.s1_token[row] = t;
+      p.a1_idx[(size_t)tb1[s] * kTileM + (row - off1[s])] = t;
+    } else {
+      myrow[k] = myrow[fk];
+    }
+    p.g.path_s1row[(size_t)t * p.K + k] = myrow[k];
+  }
+  for (int k = 0; k < p.K; ++k) {
+    const int j = rt[k];
+    if (j < 0) continue;
+    const int idx = tl * p.K + k;
+    const int r2 = off2[j] + bo2[j] + bits_below(bits2 + (size_t)j * W, idx);
+    const int q = t * p.K + k;
+    const int s = rs[k];
+    p.g.s2_path[r2] = q;
+    p.g.s2_s1row[r2] = myrow[k];
+    p.g.s2_token[r2] = t;
+    p.g.s2_w[r2] = p.w[q];
+    p.a2_idx[(size_t)tb2[j] * kTileM + (r2 - off2[j])] = tb1[s] * kTileM + (myrow[k] - off1[s]);
+  }
+}
+
+pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src, const int32_t *tgt,
+                            const float *w, const pcomoe_groups *g, char *ws, const WsLayout &lay,
+                            cudaStream_t st) {
+  const pcomoe_config &c = L->cfg;
+  GroupParams p;
+  p.src = src; p.tgt = tgt; p.w = w; p.g = *g;
+  p.plan = reinterpret_cast<DevPlan *>(ws + lay.plan);
+  p.tile_base1 = reinterpret_cast<int32_t *>(ws + lay.tile_base1);
+  p.tile_base2 = reinterpret_cast<int32_t *>(ws + lay.tile_base2);
+  p.blk_cnt = reinterpret_cast<int32_t *>(ws + lay.blk_cnt);
+  p.a1_idx = reinterpret_cast<int32_t *>(ws + lay.a1_idx);
+  p.a2_idx = reinterpret_cast<int32_t *>(ws + lay.a2_idx);
+  p.T = T; p.n = c.n_experts; p.K = c.top_k; p.dedup = c.dedup; p.chunk = L->group_chunk;
+  p.nb = (T + p.chunk - 1) / p.chunk;
+
+  // status word, plan, and the padding entries of the gather maps start from zero
+  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.plan, 0, sizeof(DevPlan), st));
+  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.a1_idx, 0, lay.u - lay.a1_idx, st));
+  count_launch(2);
+
+  const int CK = p.chunk * p.K, W = (CK + 31) / 32;
+  const size_t smem_count = sizeof(int32_t) * ((size_t)2 * CK + 2 * p.n);
+  const size_t smem_scatter = sizeof(int32_t) * ((size_t)3 * CK + 6 * p.n + (size_t)2 * p.n * W);
+  if (smem_scatter > 200 * 1024) return PCOMOE_ERR_UNSUPPORTED;
+  if (smem_count > 48 * 1024)
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(group_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_count));
+  if (smem_scatter > 48 * 1024)
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(group_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_scatter));
+  if (p.nb > 0) {
+    group_count_kernel<<<p.nb, p.chunk, smem_count, st>>>(p);
+    count_launch();
+  }
+  group_scan_kernel<<<1, 1024, 0, st>>>(p);
+  count_launch();
+  if (p.nb > 0) {
+    group_scatter_kernel<<<p.nb, p.chunk, smem_scatter, st>>>(p);
+    count_launch();
+  }
+  PCOMOE_CUDA_TRY(cudaGetLastError());
+  return PCOMOE_OK;
+}
+
+}  // namespace pcomoe

@@ -1,0 +1,239 @@
+// Host side of the C ABI: layer set-up, workspace sizing, argument checks and dispatch.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+using namespace pcomoe;
+
+namespace pcomoe {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
+  const pcomoe_config &c = L->cfg;
+  WsLayout w{};
+  const int64_t Tm = max_tokens > 0 ? max_tokens : 1;
+  const int64_t Pm = Tm * c.top_k;
+  w.nb_max = (int32_t)((Tm + L->group_chunk - 1) / L->group_chunk);
+  w.mt_max = (int32_t)(Pm / kTileM + c.n_experts + 1);
+  w.t_pad = (int32_t)((Tm + kTileM - 1) / kTileM * kTileM);
+  const size_t es = dtype_size(c.in_dtype);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align256(off + bytes);
+    return o;
+  };
+  w.plan = take(sizeof(DevPlan));
+  w.tile_base1 = take(sizeof(int32_t) * (c.n_experts + 1));
+  w.tile_base2 = take(sizeof(int32_t) * (c.n_experts + 1));
+  w.blk_cnt = take(sizeof(int32_t) * (size_t)w.nb_max * 2 * c.n_experts);
+  w.a1_idx = take(sizeof(int32_t) * (size_t)w.mt_max * kTileM);
+  w.a2_idx = take(sizeof(int32_t) * (size_t)w.mt_max * kTileM);
+  w.u = take(es * (size_t)w.mt_max * kTileM * c.ffn);
+  w.u_sh = take(es * (size_t)w.t_pad * c.shared_ffn);
+  if (L->tc_ok && !L->use_gather4) {
+    w.a_perm1 = take(es * (size_t)w.mt_max * kTileM * c.hidden);
+    w.a_perm2 = take(es * (size_t)w.mt_max * kTileM * c.ffn);
+  }
+  w.total = off;
+  return w;
+}
+
+}  // namespace pcomoe
+
+extern "C" {
+
+pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mask,
+                                  const float *h_bias, pcomoe_layer **out) {
+  if (!cfg || !h_mask || !h_bias || !out) return PCOMOE_ERR_INVALID_ARG;
+  if (cfg->struct_size != (int32_t)sizeof(pcomoe_config)) return PCOMOE_ERR_INVALID_ARG;
+  const int n = cfg->n_experts, K = cfg->top_k;
+  if (n <= 0 || K <= 0 || cfg->hidden <= 0 || cfg->ffn <= 0 || cfg->shared_ffn < 0)
+    return PCOMOE_ERR_INVALID_ARG;
+  if (cfg->in_dtype != PCOMOE_BF16 && cfg->in_dtype != PCOMOE_FP32) return PCOMOE_ERR_INVALID_ARG;
+  if (cfg->ffn_impl < PCOMOE_FFN_AUTO || cfg->ffn_impl > PCOMOE_FFN_TCGEN05)
+    return PCOMOE_ERR_INVALID_ARG;
+  if (K > n || K > kMaxTopK) return PCOMOE_ERR_SHAPE;
+  if (n > kMaxExperts) return PCOMOE_ERR_UNSUPPORTED;
+  if (cfg->out_dtype != PCOMOE_FP32) return PCOMOE_ERR_UNSUPPORTED;
+  if (cfg->hidden % 8 || cfg->ffn % 8 || cfg->shared_ffn % 8) return PCOMOE_ERR_UNSUPPORTED;
+  for (int i = 0; i < n; ++i)
+    if (!h_mask[(size_t)i * n + i]) return PCOMOE_ERR_INVALID_ARG;  // m_ii = 1 (Sec. 4.2)
+
+  pcomoe_layer *L = new (std::nothrow) pcomoe_layer();
+  if (!L) return PCOMOE_ERR_CUDA;
+  L->cfg = *cfg;
+  L->tc_ok = cfg->in_dtype == PCOMOE_BF16 && cfg->hidden % 256 == 0 && cfg->ffn % 128 == 0 &&
+             cfg->shared_ffn % 128 == 0;
+  if (cfg->ffn_impl == PCOMOE_FFN_TCGEN05 && !L->tc_ok) {
+    delete L;
+    return PCOMOE_ERR_UNSUPPORTED;
+  }
+  const char *g4 = std::getenv("PCOMOE_GATHER4");
+  L->use_gather4 = g4 ? (std::atoi(g4) != 0) : 1;
+
+  int cnt = 0;
+  for (int i = 0; i < n * n; ++i) cnt += h_mask[i] ? 1 : 0;
+  L->n_active = cnt;
+  L->h_table = (ActiveEntry *)std::malloc(sizeof(ActiveEntry) * (size_t)cnt);
+  if (!L->h_table) {
+    delete L;
+    return PCOMOE_ERR_CUDA;
+  }
+  int a = 0;
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < n; ++j)
+      if (h_mask[(size_t)i * n + j]) {
+        L->h_table[a].src = (uint16_t)i;
+        L->h_table[a].tgt = (uint16_t)j;
+        L->h_table[a].bias = h_bias[(size_t)i * n + j];
+        ++a;
+      }
+
+  // tokens per block of the grouping kernels: the two bit matrices [n][chunk*K/32] must fit
+  int chunk = 128;
+  auto scatter_smem = [&](int ch) {
+    const size_t ck = (size_t)ch * K, words = (ck + 31) / 32;
+    return 4 * (3 * ck + 6 * (size_t)n + 2 * (size_t)n * words);
+  };
+  while (chunk > 32 && scatter_smem(chunk) > 96 * 1024) chunk >>= 1;
+  L->group_chunk = chunk;
+
+  cudaError_t e = cudaGetDevice(&L->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, L->device);
+  if (e == cudaSuccess) e = cudaMalloc((void **)&L->d_table, sizeof(ActiveEntry) * (size_t)cnt);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(L->d_table, L->h_table, sizeof(ActiveEntry) * (size_t)cnt, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    if (L->d_table) cudaFree(L->d_table);
+    std::free(L->h_table);
+    delete L;
+    return PCOMOE_ERR_CUDA;
+  }
+  *out = L;
+  return PCOMOE_OK;
+}
+
+pcomoe_status pcomoe_layer_destroy(pcomoe_layer *L) {
+  if (!L) return PCOMOE_ERR_INVALID_ARG;
+  if (L->d_table) cudaFree(L->d_table);
+  std::free(L->h_table);
+  delete L;
+  return PCOMOE_OK;
+}
+
+pcomoe_status pcomoe_layer_active_set(const pcomoe_layer *L, int32_t cap, int32_t *h_src,
+                                      int32_t *h_tgt, float *h_bias, int32_t *count) {
+  if (!L || !count || cap < 0) return PCOMOE_ERR_INVALID_ARG;
+  *count = L->n_active;
+  for (int a = 0; a < L->n_active && a < cap; ++a) {
+    if (h_src) h_src[a] = L->h_table[a].src;
+    if (h_tgt) h_tgt[a] = L->h_table[a].tgt;
+    if (h_bias) h_bias[a] = L->h_table[a].bias;
+  }
+  return PCOMOE_OK;
+}
+
+pcomoe_status pcomoe_workspace_bytes(const pcomoe_layer *L, int32_t max_tokens, size_t *bytes) {
+  if (!L || !bytes || max_tokens < 0) return PCOMOE_ERR_INVALID_ARG;
+  if ((int64_t)max_tokens * L->cfg.top_k >= (int64_t)1 << 31) return PCOMOE_ERR_SHAPE;
+  *bytes = ws_layout(L, max_tokens).total;
+  return PCOMOE_OK;
+}
+
+pcomoe_status pcomoe_route_paths(const pcomoe_layer *L, int32_t T, const float *d_logits,
+                                 const float *d_tgt_logits, int32_t *d_path_src,
+                                 int32_t *d_path_tgt, float *d_path_w, void *stream) {
+  if (!L) return PCOMOE_ERR_INVALID_ARG;
+  if (T < 0) return PCOMOE_ERR_SHAPE;
+  if (T == 0) return PCOMOE_OK;
+  if (!d_logits || !d_path_src || !d_path_tgt || !d_path_w) return PCOMOE_ERR_INVALID_ARG;
+  return launch_route(L, T, d_logits, d_tgt_logits ? d_tgt_logits : d_logits, d_path_src,
+                      d_path_tgt, d_path_w, (cudaStream_t)stream);
+}
+
+static pcomoe_status check_ws(const pcomoe_layer *L, int32_t T, const void *ws, size_t ws_bytes,
+                              WsLayout *lay) {
+  if (!ws) return PCOMOE_ERR_WORKSPACE;
+  if (((uintptr_t)ws) & 255) return PCOMOE_ERR_WORKSPACE;
+  if ((int64_t)T * L->cfg.top_k >= (int64_t)1 << 31) return PCOMOE_ERR_SHAPE;
+  *lay = ws_layout(L, T);
+  if (lay->total > ws_bytes) return PCOMOE_ERR_WORKSPACE;
+  return PCOMOE_OK;
+}
+
+static bool groups_ok(const pcomoe_groups *g) {
+  return g && g->s1_offsets && g->s1_token && g->path_s1row && g->s2_offsets && g->s2_path &&
+         g->s2_s1row && g->s2_token && g->s2_w && g->stats;
+}
+
+pcomoe_status pcomoe_build_path_groups(const pcomoe_layer *L, int32_t T, const int32_t *d_path_src,
+                                       const int32_t *d_path_tgt, const float *d_path_w,
+                                       const pcomoe_groups *out, void *d_workspace, size_t ws_bytes,
+                                       void *stream) {
+  if (!L || !groups_ok(out)) return PCOMOE_ERR_INVALID_ARG;
+  if (T < 0) return PCOMOE_ERR_SHAPE;
+  if (T > 0 && (!d_path_src || !d_path_tgt || !d_path_w)) return PCOMOE_ERR_INVALID_ARG;
+  WsLayout lay;
+  pcomoe_status s = check_ws(L, T, d_workspace, ws_bytes, &lay);
+  if (s != PCOMOE_OK) return s;
+  return launch_groups(L, T, d_path_src, d_path_tgt, d_path_w, out, (char *)d_workspace, lay,
+                       (cudaStream_t)stream);
+}
+
+pcomoe_status pcomoe_ffn_forward(const pcomoe_layer *L, int32_t T, const void *d_h,
+                                 const void *d_w_gate, const void *d_w_up, const void *d_w_down,
+                                 const void *d_wsh_gate, const void *d_wsh_up,
+                                 const void *d_wsh_down, const pcomoe_groups *groups, void *d_y,
+                                 void *d_workspace, size_t ws_bytes, void *stream) {
+  if (!L || !groups_ok(groups)) return PCOMOE_ERR_INVALID_ARG;
+  if (T < 0) return PCOMOE_ERR_SHAPE;
+  if (T == 0) return PCOMOE_OK;
+  if (!d_h || !d_w_gate || !d_w_up || !d_w_down || !d_y) return PCOMOE_ERR_INVALID_ARG;
+  if (L->cfg.shared_ffn > 0 && (!d_wsh_gate || !d_wsh_up || !d_wsh_down)) return PCOMOE_ERR_INVALID_ARG;
+  WsLayout lay;
+  pcomoe_status s = check_ws(L, T, d_workspace, ws_bytes, &lay);
+  if (s != PCOMOE_OK) return s;
+  const bool tc = L->cfg.ffn_impl == PCOMOE_FFN_TCGEN05 ||
+                  (L->cfg.ffn_impl == PCOMOE_FFN_AUTO && L->tc_ok);
+  if (tc)
+    return launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
+                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream);
+  return launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
+                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream);
+}
+
+pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream) {
+  if (!d_workspace) return PCOMOE_ERR_WORKSPACE;
+  int32_t st = 0;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return PCOMOE_ERR_CUDA;
+  if (cudaMemcpy(&st, d_workspace, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return PCOMOE_ERR_CUDA;
+  if (st < 0 || st > PCOMOE_ERR_INDEX) return PCOMOE_ERR_CUDA;
+  return (pcomoe_status)st;
+}
+
+int64_t pcomoe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *pcomoe_status_string(pcomoe_status s) {
+  switch (s) {
+    case PCOMOE_OK: return "ok";
+    case PCOMOE_ERR_INVALID_ARG: return "invalid argument";
+    case PCOMOE_ERR_SHAPE: return "shape out of range";
+    case PCOMOE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case PCOMOE_ERR_UNSUPPORTED: return "unsupported size or dtype";
+    case PCOMOE_ERR_CUDA: return "CUDA call failed";
+    case PCOMOE_ERR_TIMEOUT: return "device wait timed out";
+    case PCOMOE_ERR_INDEX: return "device index out of range";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,169 @@
+// K1: compatibility-aware path routing.  One warp per token.
+//
+// For every active path a = (i,j) the warp evaluates the score of Sec. 4.2,
+//     s_a = (z[i] + b_ij) + lambda * u[j],
+// with three separately rounded fp32 operations, keeps the K best under the total order
+// (score descending, flat id ascending) - the TopK of Sec. 4.3 over the active set only -
+// and turns the selected scores into path weights with a softmax.
+#include <cfloat>
+
+#include "common.cuh"
+
+namespace pcomoe {
+
+struct RouteParams {
+  const ActiveEntry *table;  // [A], sorted by flat id, so table order == flat-id order
+  const float *z;            // [T,n]
+  const float *u;            // [T,n] (may alias z)
+  int32_t *src;              // [T,K]
+  int32_t *tgt;              // [T,K]
+  float *w;                  // [T,K]
+  int32_t T, n, K, A;
+  float lambda, scale;
+  int32_t norm_topk;
+  int32_t table_in_smem;
+};
+
+__device__ __forceinline__ float path_score(const ActiveEntry e, const float *zs, const float *us,
+                                            float lambda) {
+  float a = __fadd_rn(zs[e.src], e.bias);
+  float b = __fmul_rn(lambda, us[e.tgt]);
+  return __fadd_rn(__fadd_rn(a, b), 0.0f);  // the last add turns -0 into +0
+}
+
+// true when (s1,a1) ranks before (s2,a2)
+__device__ __forceinline__ bool ranks_before(float s1, int a1, float s2, int a2) {
+  return s1 > s2 || (s1 == s2 && a1 < a2);
+}
+
+template <int KMAX>
+__global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int warps = blockDim.x >> 5;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float *zrows = reinterpret_cast<float *>(smem_raw);                 // [warps][2][n]
+  const ActiveEntry *tab = p.table;
+  if (p.table_in_smem) {
+    ActiveEntry *st = reinterpret_cast<ActiveEntry *>(smem_raw + (((size_t)warps * 2 * p.n * 4 + 15) & ~size_t(15)));
+    for (int a = threadIdx.x; a < p.A; a += blockDim.x) st[a] = p.table[a];
+    tab = st;
+    __syncthreads();
+  }
+  float *zs = zrows + (size_t)warp * 2 * p.n;
+  float *us = zs + p.n;
+
+  for (int t = blockIdx.x * warps + warp; t < p.T; t += gridDim.x * warps) {
+    __syncwarp();
+    for (int e = lane; e < p.n; e += 32) {
+      zs[e] = p.z[(size_t)t * p.n + e];
+      us[e] = p.u[(size_t)t * p.n + e];
+    }
+    __syncwarp();
+
+    // per-lane sorted list of its best KMAX candidates (ties keep the smaller table index first,
+    // because a lane visits its entries in ascending order and only a strictly larger score moves up)
+    float ls[KMAX];
+    int la[KMAX];
+#pragma unroll
+    for (int i = 0; i < KMAX; ++i) {
+      ls[i] = -FLT_MAX;
+      la[i] = 0x7fffffff;
+    }
+    for (int a = lane; a < p.A; a += 32) {
+      const float s = path_score(tab[a], zs, us, p.lambda);
+      if (s > ls[KMAX - 1] || la[KMAX - 1] == 0x7fffffff) {
+        ls[KMAX - 1] = s;
+        la[KMAX - 1] = a;
+#pragma unroll
+        for (int i = KMAX - 1; i > 0; --i) {
+          if (ranks_before(ls[i], la[i], ls[i - 1], la[i - 1])) {
+            float ts = ls[i]; ls[i] = ls[i - 1]; ls[i - 1] = ts;
+            int ta = la[i]; la[i] = la[i - 1]; la[i - 1] = ta;
+          }
+        }
+      }
+    }
+
+    // K rounds of warp arg-max over the lane heads
+    float my_s = -FLT_MAX;
+    int my_a = 0;
+    for (int k = 0; k < p.K; ++k) {
+      float bs = ls[0];
+      int ba = la[0];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        const float os = __shfl_xor_sync(0xffffffffu, bs, off);
+        const int oa = __shfl_xor_sync(0xffffffffu, ba, off);
+        if (ranks_before(os, oa, bs, ba)) {
+          bs = os;
+          ba = oa;
+        }
+      }
+      if (la[0] == ba) {  // this lane owns the winner: pop it
+#pragma unroll
+        for (int i = 0; i < KMAX - 1; ++i) {
+          ls[i] = ls[i + 1];
+          la[i] = la[i + 1];
+        }
+        ls[KMAX - 1] = -FLT_MAX;
+        la[KMAX - 1] = 0x7fffffff;
+      }
+      if (lane == k) {
+        my_s = bs;
+        my_a = ba;
+      }
+    }
+
+    const float s0 = __shfl_sync(0xffffffffu, my_s, 0);
+    float e = lane < p.K ? expf(my_s - s0) : 0.0f;
+    float den;
+    if (p.norm_topk) {
+      den = e;
+    } else {
+      den = 0.0f;
+      for (int a = lane; a < p.A; a += 32) den += expf(path_score(tab[a], zs, us, p.lambda) - s0);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
+    if (lane < p.K) {
+      const ActiveEntry en = tab[my_a];
+      const size_t o = (size_t)t * p.K + lane;
+      p.src[o] = en.src;
+      p.tgt[o] = en.tgt;
+      p.w[o] = e / den * p.scale;
+    }
+  }
+}
+
+pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, const float *u,
+                           int32_t *src, int32_t *tgt, float *w, cudaStream_t st) {
+  const pcomoe_config &c = L->cfg;
+  RouteParams p;
+  p.table = L->d_table;
+  p.z = z; p.u = u; p.src = src; p.tgt = tgt; p.w = w;
+  p.T = T; p.n = c.n_experts; p.K = c.top_k; p.A = L->n_active;
+  p.lambda = c.lambda; p.scale = c.routed_scale; p.norm_topk = c.norm_topk;
+  const int threads = 256, warps = threads / 32;
+  size_t smem = ((size_t)warps * 2 * p.n * 4 + 15) & ~size_t(15);
+  const size_t tab_bytes = sizeof(ActiveEntry) * (size_t)p.A;
+  p.table_in_smem = smem + tab_bytes <= 160 * 1024;
+  if (p.table_in_smem) smem += tab_bytes;
+  int grid = (T + warps - 1) / warps;
+  const int cap = L->sm_count * 4;
+  if (grid > cap) grid = cap;
+
+  void (*kern)(const RouteParams) = nullptr;
+  if (p.K <= 2) kern = route_kernel<2>;
+  else if (p.K <= 4) kern = route_kernel<4>;
+  else if (p.K <= 8) kern = route_kernel<8>;
+  else if (p.K <= 16) kern = route_kernel<16>;
+  else kern = route_kernel<32>;
+  if (smem > 48 * 1024)
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<grid, threads, smem, st>>>(p);
+  count_launch();
+  PCOMOE_CUDA_TRY(cudaGetLastError());
+  return PCOMOE_OK;
+}
+
+}  // namespace pcomoe
