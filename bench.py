@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the path-composed MoE FFN layer: one step = one pass of the whole hot path
+(route -> group -> stage 1 -> stage 2) over one batch of seeded synthetic tokens.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is tokens/s over all ranks with inputs resident in HBM;
+`e2e` is the same metric through the host-buffer call (pinned H2D of logits and hidden states, D2H
+of y inside the timed region); `roofline` covers the dominant kernel (stage-1 grouped GEMM) timed
+alone with CUDA events; `cpu_baseline` is the CPU oracle timed on a bounded token sample.
+With --impl reference the CPU oracle itself is the timed arm (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_01024_b200 import workloads as wl  # noqa: E402
+
+METRIC = "path_moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.rows:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v == "Active":
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_work(cfg, R1, n_src, n_tgt):
+    """FLOPs and bytes the method must do for one layer call (deduplicated stage 1, weights of the
+    touched experts once, activations once)."""
+    P = cfg.T * cfg.K
+    H, F, Fs, T = cfg.H, cfg.F, cfg.F_sh, cfg.T
+    es = 4 if cfg.dtype == "f32" else 2
+    flops_s1 = 4.0 * R1 * H * F
+    flops_s2 = 2.0 * P * H * F
+    flops_sh = 6.0 * T * H * Fs
+    wbytes = es * ((2 * n_src + n_tgt) * H * F + 3 * H * Fs)
+    abytes = es * T * H + es * R1 * F + es * P * F + 4 * T * H + 4 * T * cfg.n + 36 * P + (2 * es * T * Fs)
+    return dict(flops=flops_s1 + flops_s2 + flops_sh, flops_s1=flops_s1, flops_s2=flops_s2, flops_sh=flops_sh,
+                bytes=wbytes + abytes, weight_bytes=wbytes)
+
+
+def oracle_sample_rate(cfg, L, n_tok, seed=0):
+    """Times the CPU oracle (routing + grouping on all tokens, FFN on a seeded sample of n_tok tokens).
+    Returns (tokens/s of the FFN sample incl. the per-token share of routing, threads, seconds)."""
+    import oracle
+    oracle.build()
+    hf = wl.hidden_as_f32(cfg, L.h)
+    t0 = time.time()
+    src, tgt, w = oracle.route(L.logits, L.mask, L.bias, cfg.lam, cfg.K)
+    oracle.groups(src, tgt, w, cfg.n)
+    t_route = time.time() - t0
+    rng = np.random.default_rng(seed)
+    toks = np.sort(rng.choice(cfg.T, size=min(n_tok, cfg.T), replace=False)).astype(np.int32)
+    shared = (L.wsh_gate, L.wsh_up, L.wsh_down) if cfg.F_sh else None
+    t0 = time.time()
+    oracle.ffn(hf, L.w_gate, L.w_up, L.w_down, src, tgt, w, shared=shared, tokens=toks)
+    t_ffn = time.time() - t0
+    per_tok = t_ffn / len(toks) + t_route / cfg.T
+    return 1.0 / per_tok, oracle.threads(), t_ffn + t_route, len(toks)
+
+
+def run_reference(args, cfg):
+    """The CPU oracle as the timed arm: each step evaluates a bounded token sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    L = wl.make_layer(cfg)
+    n_tok = args.ref_tokens
+    rates, secs = [], []
+    for i in range(args.warmup + args.steps):
+        r, thr, s, nt = oracle_sample_rate(cfg, L, n_tok, seed=i)
+        if i >= args.warmup:
+            rates.append(r); secs.append(s)
+    v = statistics.mean(rates)
+    sample = f"routing+grouping on all {cfg.T} tokens, FFN on {nt} seeded tokens per step"
+    out = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": 1e3 * cfg.T / v, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "F": cfg.F, "n": cfg.n, "K": cfg.K,
+                      "F_sh": cfg.F_sh, "sample": sample},
+           "cpu_baseline": {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
+           "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=2, help="benchmark layer 1..5 (2 = the configuration the metric is quoted on)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-tokens", type=int, default=0,
+                    help="tokens of the CPU-oracle sample (0: sized for roughly 15 s from a short probe)")
+    ap.add_argument("--shape", default=None,
+                    help="T,H,F,n,K,F_sh: a reduced layer with the recipe of --config (for profiler captures)")
+    ap.add_argument("--profile", action="store_true",
+                    help="only run warm-up + steps of the device-resident hot path, print a short line and exit")
+    ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--variant", default="default", choices=["default", "vanilla"],
+                    help="vanilla: diagonal-only mask (every path a whole expert, no reuse)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = wl.CONFIGS[args.config]
+    if args.shape:
+        T, H, F, n, K, Fs = (int(x) for x in args.shape.split(","))
+        cfg = cfg.scaled(name=f"{cfg.name}-reduced-T{T}-H{H}-F{F}-n{n}-K{K}-Fsh{Fs}", T=T, H=H, F=F, n=n, K=K, F_sh=Fs)
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_01024_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    # Every rank holds a replica of the weights and its own batch of T tokens (token data parallel,
+    # no collective on the data path); rank r draws its tokens with seed + 100*r.
+    cfg_r = cfg if rank == 0 else cfg.scaled(seed=cfg.seed)  # same weights on every rank
+    L = wl.make_layer(cfg_r)
+    if rank > 0:
+        cfg_tok = cfg.scaled(seed=cfg.seed + 100 * rank)
+        L.h = wl.make_hidden(cfg_tok)
+        L.logits = wl.make_logits(cfg_tok, wl.hidden_as_f32(cfg_tok, L.h) if cfg.logits == "router" else None)
+    mask = np.eye(cfg.n, dtype=np.uint8) if args.variant == "vanilla" else L.mask
+    dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
+    layer = B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=cfg.F, mask=mask, bias=L.bias,
+                           w_gate=B.to_device(L.w_gate, dev), w_up=B.to_device(L.w_up, dev),
+                           w_down=B.to_device(L.w_down, dev),
+                           shared=tuple(B.to_device(x, dev) for x in (L.wsh_gate, L.wsh_up, L.wsh_down)) if cfg.F_sh else None,
+                           max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam, device=dev)
+    d_logits = torch.from_numpy(L.logits).to(dev)
+    d_h = B.to_device(L.h, dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps ----
+    for _ in range(args.warmup):
+        layer.forward(d_logits, d_h)
+    assert layer.device_status() == 0, "device reported an error during warm-up"
+    if args.profile:
+        for _ in range(args.steps):
+            layer.forward(d_logits, d_h)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_run": cfg.name, "steps": args.steps, "status": layer.device_status()}))
+        return
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    n0 = B.pcomoe_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        layer.forward(d_logits, d_h)
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = B.pcomoe_launch_count() - n0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    assert layer.device_status() == 0, "device reported an error during the timed steps"
+    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_max = float(t_ms.item())
+    ms_per_step = ms_max / args.steps
+    value = world * cfg.T / (ms_per_step * 1e-3)
+
+    # ---- end to end through host buffers (pinned H2D of inputs, D2H of y) ----
+    for _ in range(2):
+        layer.forward_host(L.logits, L.h)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        y_host = layer.forward_host(L.logits, L.h)
+    torch.cuda.synchronize()
+    t_e2e = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
+    e2e_value = world * cfg.T * args.steps / float(t_e2e.item())
+    h2d = L.logits.nbytes + L.h.nbytes
+    d2h = cfg.T * cfg.H * 4
+
+    # ---- per-kernel timing for the roofline: dominant kernel = stage-1 grouped GEMM ----
+    stats = layer.groups.stats.cpu().numpy()
+    R1 = int(stats[0])
+    n_src = cfg.n - int(stats[4]); n_tgt = cfg.n - int(stats[5])
+    work = algorithmic_work(cfg, R1, n_src, n_tgt)
+    stage_ms = {}
+    for name, fn in (("route", lambda: layer.route(d_logits)), ("groups", lambda: layer.build_groups(cfg.T)),
+                     ("stage1_routed", lambda: layer.ffn_stages(d_h, 1)), ("stage1_shared", lambda: layer.ffn_stages(d_h, 2)),
+                     ("stage2_routed", lambda: layer.ffn_stages(d_h, 4)), ("stage2_shared", lambda: layer.ffn_stages(d_h, 8))):
+        if "shared" in name and not cfg.F_sh:
+            continue
+        ts = []
+        for i in range(3 + args.steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        stage_ms[name] = statistics.mean(ts)
+    pk = peaks()
+    tc_path = cfg.dtype == "bf16"
+    if tc_path and cfg.T >= 1024:
+        # prefill-sized: tensor-bound; stage-1 routed GEMM is the dominant kernel
+        ach = work["flops_s1"] / (stage_ms["stage1_routed"] * 1e-3) / 1e12
+        peak = pk["bf16_tflops_sustained"]
+        roofline = {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                    "traffic": None, "kernel": "grouped_gemm_kernel<1> (stage 1, routed groups)",
+                    "peak_source": pk["source"] + " sustained bf16 (kernel timed inside a loop of steps)"}
+    else:
+        # decode-sized / tiny: weight streaming; report the two GEMM stages' bytes against HBM
+        s1_bytes = 2 * (2 * n_src * cfg.H * cfg.F) if tc_path else 4 * (2 * n_src * cfg.H * cfg.F)
+        ach = s1_bytes / (stage_ms["stage1_routed"] * 1e-3) / 1e9
+        peak = pk["hbm_gbs"]
+        roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                    "traffic": None, "kernel": "stage 1, routed groups (weight streaming)",
+                    "peak_source": pk["source"] + " copy bandwidth"}
+    # whole-layer roofline time: max(FLOPs / tensor peak, bytes / HBM peak)
+    t_roof_meas = max(work["flops"] / (pk["bf16_tflops_sustained"] * 1e12), work["bytes"] / (pk["hbm_gbs"] * 1e9))
+    t_roof_nominal = max(work["flops"] / 2.25e15, work["bytes"] / 8e12)
+
+    out = None
+    if rank == 0:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16" if tc_path else "f32", "data": "synthetic",
+               "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
+                          "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam,
+                          "R1_over_P": R1 / (cfg.T * cfg.K), "parallelism": f"token-dp{world} (replicas, no collective)",
+                          "l2": "inputs larger than L2 (weights are streamed every step)" if work["weight_bytes"] > 126e6
+                                else "working set fits L2; not a performance target"},
+               "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+               "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+               "layer_roofline": {"flops": work["flops"], "bytes": work["bytes"],
+                                  "frac_of_measured": t_roof_meas / (ms_per_step * 1e-3),
+                                  "frac_of_nominal_2.25PF_8TBs": t_roof_nominal / (ms_per_step * 1e-3)},
+               "stage_ms": stage_ms}
+        if not args.no_cpu_baseline and world == 1:
+            n_cpu = args.cpu_tokens
+            if n_cpu <= 0:   # probe with a few tokens, then size the sample for about 15 s
+                r0, _, s0, nt0 = oracle_sample_rate(cfg, L, 8)
+                n_cpu = int(max(8, min(cfg.T, 15.0 * r0)))
+            r, thr, secs, nt = oracle_sample_rate(cfg, L, n_cpu)
+            out["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": thr, "kind": "oracle",
+                                   "sample": f"routing+grouping on all {cfg.T} tokens, FFN on {nt} seeded tokens ({secs:.1f} s)"}
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -164,6 +164,17 @@ pcomoe_status pcomoe_ffn_forward(const pcomoe_layer *layer, int32_t T, const voi
                                  const void *d_wsh_down, const pcomoe_groups *groups, void *d_y,
                                  void *d_workspace, size_t ws_bytes, void *stream);
 
+/* The pieces of pcomoe_ffn_forward one by one, for timing and for checking a stage alone (same
+ * arguments and errors).  `stages` is a bit mask: 1 = stage 1 over the routed groups, 2 = stage 1 of
+ * the shared expert, 4 = zero-fill of y and stage 2 over the routed groups, 8 = stage 2 of the shared
+ * expert.  pcomoe_ffn_forward is stages = 15.  Stage 2 reads what stage 1 left in the workspace. */
+pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, const void *d_h,
+                                        const void *d_w_gate, const void *d_w_up,
+                                        const void *d_w_down, const void *d_wsh_gate,
+                                        const void *d_wsh_up, const void *d_wsh_down,
+                                        const pcomoe_groups *groups, void *d_y, void *d_workspace,
+                                        size_t ws_bytes, void *stream, int32_t stages);
+
 /* Synchronises `stream`, reads the workspace's status word and returns the first error a kernel
  * recorded (PCOMOE_OK if none); the word is cleared by the next pcomoe_build_path_groups. */
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream);

@@ -21,7 +21,8 @@ PCOMOE_BF16, PCOMOE_FP32 = 0, 1
 PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
-           "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_ffn_forward", "pcomoe_device_status",
+           "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_ffn_forward", "pcomoe_ffn_forward_stages",
+           "pcomoe_device_status",
            "pcomoe_launch_count", "pcomoe_status_string"]
 
 
@@ -64,6 +65,7 @@ def load_library(path: str | None = None):
     lib.pcomoe_route_paths.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.pcomoe_build_path_groups.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, sz, vp]
     lib.pcomoe_ffn_forward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
+    lib.pcomoe_ffn_forward_stages.argtypes = lib.pcomoe_ffn_forward.argtypes + [i32]
     lib.pcomoe_device_status.argtypes = [vp, vp]
     lib.pcomoe_launch_count.restype = ctypes.c_int64
     lib.pcomoe_status_string.restype = ctypes.c_char_p
@@ -175,6 +177,15 @@ def pcomoe_ffn_forward(layer, T, h, w_gate, w_up, w_down, wsh_gate, wsh_up, wsh_
                                              _stream()), "pcomoe_ffn_forward")
 
 
+def pcomoe_ffn_forward_stages(layer, T, h, w_gate, w_up, w_down, wsh_gate, wsh_up, wsh_down, groups: Groups, y,
+                              workspace, stages: int):
+    _check(load_library().pcomoe_ffn_forward_stages(layer, T, _ptr(h), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                                                    _ptr(wsh_gate), _ptr(wsh_up), _ptr(wsh_down),
+                                                    ctypes.byref(groups.c), _ptr(y), _ptr(workspace),
+                                                    workspace.numel() * workspace.element_size(), _stream(),
+                                                    stages), "pcomoe_ffn_forward_stages")
+
+
 def pcomoe_device_status(workspace) -> int:
     return int(load_library().pcomoe_device_status(_ptr(workspace), _stream()))
 
@@ -232,6 +243,11 @@ class PathMoELayer:
         T = h.shape[0]
         pcomoe_ffn_forward(self.layer, T, h, self.w_gate, self.w_up, self.w_down, *self.shared, self.groups,
                            self.y, self.workspace)
+
+    def ffn_stages(self, h, stages: int):
+        T = h.shape[0]
+        pcomoe_ffn_forward_stages(self.layer, T, h, self.w_gate, self.w_up, self.w_down, *self.shared, self.groups,
+                                  self.y, self.workspace, stages)
 
     def forward(self, logits, h, tgt_logits=None):
         """The whole hot path on device tensors: route -> group -> stage 1 -> stage 2.  Returns y [T,H] fp32."""

@@ -86,10 +86,13 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
 pcomoe_status launch_ffn_simt(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                               const void *wu, const void *wd, const void *sg, const void *su,
                               const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                              const WsLayout &lay, cudaStream_t st);
+                              const WsLayout &lay, cudaStream_t st, int stages);
 pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                             const void *wu, const void *wd, const void *sg, const void *su,
                             const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                            const WsLayout &lay, cudaStream_t st);
+                            const WsLayout &lay, cudaStream_t st, int stages);
+
+// bits of `stages`
+constexpr int kStage1Routed = 1, kStage1Shared = 2, kStage2Routed = 4, kStage2Shared = 8;
 
 }  // namespace pcomoe

@@ -114,39 +114,46 @@ template <typename E>
 static pcomoe_status run_simt(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                               const void *wu, const void *wd, const void *sg, const void *su,
                               const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                              const WsLayout &lay, cudaStream_t st) {
+                              const WsLayout &lay, cudaStream_t st, int stages) {
   const pcomoe_config &c = L->cfg;
   DevPlan *plan = reinterpret_cast<DevPlan *>(ws + lay.plan);
   E *U = reinterpret_cast<E *>(ws + lay.u);
   E *Ush = reinterpret_cast<E *>(ws + lay.u_sh);
   const int P = T * c.top_k;
-  PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * c.hidden, st));
-  count_launch();
-
   SimtArgs a1{};
   a1.offsets = g->s1_offsets; a1.row_src = g->s1_token; a1.G = c.n_experts; a1.rows = P;
   a1.H = c.hidden; a1.F = c.ffn; a1.limit_src = T; a1.T = T; a1.plan = plan;
   const int gy1 = max(1, min(16, c.ffn / 64));
-  simt_stage1_kernel<E><<<dim3(P, gy1), 128, sizeof(float) * c.hidden, st>>>(
-      a1, (const E *)h, (const E *)wg, (const E *)wu, U);
-  count_launch();
+  if (stages & kStage1Routed) {
+    simt_stage1_kernel<E><<<dim3(P, gy1), 128, sizeof(float) * c.hidden, st>>>(
+        a1, (const E *)h, (const E *)wg, (const E *)wu, U);
+    count_launch();
+  }
 
   SimtArgs a2{};
   a2.offsets = g->s2_offsets; a2.row_src = g->s2_s1row; a2.row_token = g->s2_token; a2.row_w = g->s2_w;
   a2.G = c.n_experts; a2.rows = P; a2.H = c.hidden; a2.F = c.ffn; a2.limit_src = P; a2.T = T; a2.plan = plan;
   const int gy2 = max(1, min(16, c.hidden / 64));
-  simt_stage2_kernel<E><<<dim3(P, gy2), 128, sizeof(float) * c.ffn, st>>>(a2, U, (const E *)wd, y);
-  count_launch();
+  if (stages & kStage2Routed) {
+    PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * c.hidden, st));
+    simt_stage2_kernel<E><<<dim3(P, gy2), 128, sizeof(float) * c.ffn, st>>>(a2, U, (const E *)wd, y);
+    count_launch(2);
+  }
 
   if (c.shared_ffn > 0) {
     SimtArgs s1{};
     s1.G = 1; s1.rows = T; s1.H = c.hidden; s1.F = c.shared_ffn; s1.limit_src = T; s1.T = T; s1.plan = plan;
     const int gy = max(1, min(16, c.shared_ffn / 64));
-    simt_stage1_kernel<E><<<dim3(T, gy), 128, sizeof(float) * c.hidden, st>>>(
-        s1, (const E *)h, (const E *)sg, (const E *)su, Ush);
+    if (stages & kStage1Shared) {
+      simt_stage1_kernel<E><<<dim3(T, gy), 128, sizeof(float) * c.hidden, st>>>(
+          s1, (const E *)h, (const E *)sg, (const E *)su, Ush);
+      count_launch();
+    }
     SimtArgs s2 = s1;
-    simt_stage2_kernel<E><<<dim3(T, gy2), 128, sizeof(float) * c.shared_ffn, st>>>(s2, Ush, (const E *)sd, y);
-    count_launch(2);
+    if (stages & kStage2Shared) {
+      simt_stage2_kernel<E><<<dim3(T, gy2), 128, sizeof(float) * c.shared_ffn, st>>>(s2, Ush, (const E *)sd, y);
+      count_launch();
+    }
   }
   PCOMOE_CUDA_TRY(cudaGetLastError());
   return PCOMOE_OK;
@@ -155,7 +162,7 @@ static pcomoe_status run_simt(const pcomoe_layer *L, int32_t T, const void *h, c
 pcomoe_status launch_ffn_simt(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                               const void *wu, const void *wd, const void *sg, const void *su,
                               const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                              const WsLayout &lay, cudaStream_t st) {
+                              const WsLayout &lay, cudaStream_t st, int stages) {
   const size_t need = sizeof(float) * (size_t)max(max(L->cfg.hidden, L->cfg.ffn), L->cfg.shared_ffn);
   if (need > 200 * 1024) return PCOMOE_ERR_UNSUPPORTED;
   if (need > 48 * 1024) {
@@ -165,8 +172,8 @@ pcomoe_status launch_ffn_simt(const pcomoe_layer *L, int32_t T, const void *h, c
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(simt_stage2_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need));
   }
   if (L->cfg.in_dtype == PCOMOE_FP32)
-    return run_simt<float>(L, T, h, wg, wu, wd, sg, su, sd, g, y, ws, lay, st);
-  return run_simt<__nv_bfloat16>(L, T, h, wg, wu, wd, sg, su, sd, g, y, ws, lay, st);
+    return run_simt<float>(L, T, h, wg, wu, wd, sg, su, sd, g, y, ws, lay, st, stages);
+  return run_simt<__nv_bfloat16>(L, T, h, wg, wu, wd, sg, su, sd, g, y, ws, lay, st, stages);
 }
 
 }  // namespace pcomoe

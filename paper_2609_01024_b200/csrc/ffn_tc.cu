@@ -438,7 +438,7 @@ constexpr size_t kSmemDyn = (size_t)STAGES * STAGE_BYTES + 1024;
 pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                             const void *wu, const void *wd, const void *sg, const void *su,
                             const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                            const WsLayout &lay, cudaStream_t st) {
+                            const WsLayout &lay, cudaStream_t st, int stages) {
   const pcomoe_config &c = L->cfg;
   if (!L->tc_ok) return PCOMOE_ERR_UNSUPPORTED;
   const int n = c.n_experts, H = c.hidden, F = c.ffn, Fsh = c.shared_ffn;
@@ -465,8 +465,10 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   if (!L->use_gather4) {
     // gather-free fallback: rows are first copied into the padded order, then loaded as plain tiles
     uint4 *p1 = reinterpret_cast<uint4 *>(ws + lay.a_perm1);
-    gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(p1, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
-    count_launch();
+    if (stages & kStage1Routed) {
+      gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(p1, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
+      count_launch();
+    }
     a1_src = p1;
     a2_src = ws + lay.a_perm2;
     ok = ok && make_map(&mA1, a1_src, pad_rows, H, kTileM);
@@ -480,16 +482,15 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   ok = ok && make_map(&mD, wd, (uint64_t)n * H, F, 256);
   if (!ok) return PCOMOE_ERR_CUDA;
 
-  PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * H, st));
-  count_launch();
-
   const int grid = L->sm_count;
   TcParams p1{};
   p1.tile_base = tb1; p1.row_offsets = g->s1_offsets; p1.a_idx = L->use_gather4 ? a1 : nullptr;
   p1.G = n; p1.nt = F / 128; p1.kb = H / BK; p1.b_group_rows = F;
   p1.u_out = U; p1.ldu = F; p1.T = T; p1.plan = plan;
-  grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA1, mG, mU, p1);
-  count_launch();
+  if (stages & kStage1Routed) {
+    grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA1, mG, mU, p1);
+    count_launch();
+  }
 
   CUtensorMap mHs, mSg, mSu, mUs, mSd;
   if (Fsh > 0) {
@@ -500,11 +501,13 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     TcParams s1{};
     s1.G = 1; s1.single_rows = T; s1.nt = Fsh / 128; s1.kb = H / BK; s1.b_group_rows = 0;
     s1.u_out = Ush; s1.ldu = Fsh; s1.T = T; s1.plan = plan;
-    grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mHs, mSg, mSu, s1);
-    count_launch();
+    if (stages & kStage1Shared) {
+      grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mHs, mSg, mSu, s1);
+      count_launch();
+    }
   }
 
-  if (!L->use_gather4) {
+  if (!L->use_gather4 && (stages & kStage2Routed)) {
     uint4 *p2 = reinterpret_cast<uint4 *>(ws + lay.a_perm2);
     gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(p2, reinterpret_cast<const uint4 *>(U), a2, tb2, n, F / 8);
     count_launch();
@@ -513,10 +516,13 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   p2.tile_base = tb2; p2.row_offsets = g->s2_offsets; p2.a_idx = L->use_gather4 ? a2 : nullptr;
   p2.G = n; p2.nt = H / 256; p2.kb = F / BK; p2.b_group_rows = H;
   p2.row_token = g->s2_token; p2.row_w = g->s2_w; p2.y = y; p2.ldy = H; p2.T = T; p2.plan = plan;
-  grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA2, mD, mD, p2);
-  count_launch();
+  if (stages & kStage2Routed) {
+    PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * H, st));
+    grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA2, mD, mD, p2);
+    count_launch(2);
+  }
 
-  if (Fsh > 0) {
+  if (Fsh > 0 && (stages & kStage2Shared)) {
     TcParams s2{};
     s2.G = 1; s2.single_rows = T; s2.nt = H / 256; s2.kb = Fsh / BK; s2.b_group_rows = 0;
     s2.y = y; s2.ldy = H; s2.T = T; s2.plan = plan;

@@ -77,7 +77,7 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
     return PCOMOE_ERR_UNSUPPORTED;
   }
   const char *g4 = std::getenv("PCOMOE_GATHER4");
-  L->use_gather4 = g4 ? (std::atoi(g4) != 0) : 1;
+  L->use_gather4 = g4 ? (std::atoi(g4) != 0) : 0;
 
   int cnt = 0;
   for (int i = 0; i < n * n; ++i) cnt += h_mask[i] ? 1 : 0;
@@ -193,7 +193,17 @@ pcomoe_status pcomoe_ffn_forward(const pcomoe_layer *L, int32_t T, const void *d
                                  const void *d_wsh_gate, const void *d_wsh_up,
                                  const void *d_wsh_down, const pcomoe_groups *groups, void *d_y,
                                  void *d_workspace, size_t ws_bytes, void *stream) {
-  if (!L || !groups_ok(groups)) return PCOMOE_ERR_INVALID_ARG;
+  return pcomoe_ffn_forward_stages(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up,
+                                   d_wsh_down, groups, d_y, d_workspace, ws_bytes, stream, 15);
+}
+
+pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *L, int32_t T, const void *d_h,
+                                        const void *d_w_gate, const void *d_w_up,
+                                        const void *d_w_down, const void *d_wsh_gate,
+                                        const void *d_wsh_up, const void *d_wsh_down,
+                                        const pcomoe_groups *groups, void *d_y, void *d_workspace,
+                                        size_t ws_bytes, void *stream, int32_t stages) {
+  if (!L || !groups_ok(groups) || stages < 0 || stages > 15) return PCOMOE_ERR_INVALID_ARG;
   if (T < 0) return PCOMOE_ERR_SHAPE;
   if (T == 0) return PCOMOE_OK;
   if (!d_h || !d_w_gate || !d_w_up || !d_w_down || !d_y) return PCOMOE_ERR_INVALID_ARG;
@@ -205,9 +215,9 @@ pcomoe_status pcomoe_ffn_forward(const pcomoe_layer *L, int32_t T, const void *d
                   (L->cfg.ffn_impl == PCOMOE_FFN_AUTO && L->tc_ok);
   if (tc)
     return launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
-                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream);
+                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
   return launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
-                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream);
+                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
 }
 
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream) {
