@@ -146,6 +146,43 @@ pcomoe_status pcomoe_build_path_groups(const pcomoe_layer *layer, int32_t T,
                                        void *d_workspace, size_t ws_bytes, void *stream);
 
 /*
+ * The grouping step for callers that cannot provide a workspace.  (No counterpart in the paper: this
+ * entry point exists for deployment reasons only.)
+ *
+ * Who needs it: code that must group paths but has no means of getting device memory when it runs -
+ * for instance a routing component loaded into a serving process after the engine has reserved the
+ * whole GPU for its own pools, or a host application that forbids allocation (and the device-wide
+ * synchronisation an allocation or a free implies) on its request path.  Such a caller still owns its
+ * inputs and outputs; what it lacks is the scratch that pcomoe_build_path_groups takes from
+ * d_workspace.  This variant keeps that scratch in a fixed array of PCOMOE_STATIC_SCRATCH_BYTES inside
+ * the library's device image (every GPU on which the library is used holds the array until the
+ * process exits) and calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Same inputs, outputs, order and results as pcomoe_build_path_groups (the group arrays in `out` are
+ * bit-identical).  The tile schedule and gather maps it leaves behind are in the internal array, not in
+ * a workspace, so pcomoe_ffn_forward cannot follow this call; use it when the group arrays themselves
+ * are what is needed.
+ *
+ * Limits and rules:
+ *   - The layer must have been created on the current device (else INVALID_ARG).
+ *   - The scratch need grows with T*K and n; T*K <= 65536 always fits (n <= 256).  A larger batch
+ *     that does not fit is refused with PCOMOE_ERR_SHAPE and nothing is enqueued.
+ *   - The first call on a device looks up the array's device address (a one-time set-up for that
+ *     device); make that first call before any stream capture begins.
+ *   - Every call on a device uses the same array.  Each call zero-fills what must start from zero,
+ *     so nothing is carried over from the previous call, but two calls that can run on the GPU at
+ *     the same time (different streams) race: serialise them.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED (device ordinal >= 64), CUDA.  Device: INDEX, recorded in
+ * the internal status word only (not readable through pcomoe_device_status); rows of an
+ * out-of-range expert id are skipped.
+ */
+#define PCOMOE_STATIC_SCRATCH_BYTES (2u << 20)
+pcomoe_status pcomoe_build_path_groups_static(const pcomoe_layer *layer, int32_t T,
+                                              const int32_t *d_path_src, const int32_t *d_path_tgt,
+                                              const float *d_path_w, const pcomoe_groups *out,
+                                              void *stream);
+
+/*
  * Layer forward over the groups (Sec. 4.1 operators U_e, D_e; Sec. 4.3 source-grouped output):
  *   stage 1  for each source i and each of its rows r:  U[r,:] = SiLU(W_gate^(i) h_t) (.) (W_up^(i) h_t),
  *            t = s1_token[r]                 (bf16 storage: fp32 accumulate, U kept in bf16)

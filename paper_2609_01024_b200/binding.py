@@ -21,7 +21,8 @@ PCOMOE_BF16, PCOMOE_FP32 = 0, 1
 PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
-           "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_ffn_forward", "pcomoe_ffn_forward_stages",
+           "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",
+           "pcomoe_ffn_forward_stages",
            "pcomoe_device_status",
            "pcomoe_launch_count", "pcomoe_status_string"]
 
@@ -64,6 +65,7 @@ def load_library(path: str | None = None):
     lib.pcomoe_workspace_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
     lib.pcomoe_route_paths.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.pcomoe_build_path_groups.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, sz, vp]
+    lib.pcomoe_build_path_groups_static.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp]
     lib.pcomoe_ffn_forward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
     lib.pcomoe_ffn_forward_stages.argtypes = lib.pcomoe_ffn_forward.argtypes + [i32]
     lib.pcomoe_device_status.argtypes = [vp, vp]
@@ -168,6 +170,14 @@ def pcomoe_build_path_groups(layer, T, path_src, path_tgt, path_w, groups: Group
                                                    ctypes.byref(groups.c), _ptr(workspace),
                                                    workspace.numel() * workspace.element_size(), _stream()),
            "pcomoe_build_path_groups")
+
+
+def pcomoe_build_path_groups_static(layer, T, path_src, path_tgt, path_w, groups: Groups) -> int:
+    """Grouping without a workspace, for callers that cannot allocate one: the scratch is a fixed
+    array inside the library.  Returns the pcomoe_status instead of raising, so that a refusal
+    (batch too large for the fixed array) can be inspected."""
+    return int(load_library().pcomoe_build_path_groups_static(layer, T, _ptr(path_src), _ptr(path_tgt),
+                                                              _ptr(path_w), ctypes.byref(groups.c), _stream()))
 
 
 def pcomoe_ffn_forward(layer, T, h, w_gate, w_up, w_down, wsh_gate, wsh_up, wsh_down, groups: Groups, y, workspace):
