@@ -38,12 +38,13 @@ struct WsLayout {
   size_t tile_base1;   // int32 [n+1]   prefix of stage-1 m-tiles per source
   size_t tile_base2;   // int32 [n+1]   prefix of stage-2 m-tiles per target
   size_t blk_cnt;      // int32 [NB][2][n] per-block histograms, turned into offsets by the scan
-  size_t a1_idx;       // int32 [mt_max*128] token of every padded stage-1 row
-  size_t a2_idx;       // int32 [mt_max*128] padded U row of every padded stage-2 row
-  size_t u;            // in_dtype [mt_max*128, F]   intermediates, groups padded to 128 rows
+  size_t a1_idx;       // int32 [mt_max*128] token of every padded stage-1 row (0 in the padding)
+  size_t path_prow1;   // int32 [T*K] padded stage-1 row of every path
+  size_t path_pos2;    // int32 [T*K] padded stage-2 row of every path
+  size_t u;            // in_dtype [mt_max*128, F]   intermediates (tensor-core path: in padded stage-2
+                       //                            order; SIMT path: by unpadded stage-1 row)
   size_t u_sh;         // in_dtype [Tpad, F_sh]      shared-expert intermediates
-  size_t a_perm1;      // bf16 [mt_max*128, H]  (only when the gather-free fallback is enabled)
-  size_t a_perm2;      // bf16 [mt_max*128, F]
+  size_t h_gath;       // bf16 [mt_max*128, H]       rows of h in padded stage-1 order (tensor-core path)
   size_t total;
   int32_t nb_max;      // blocks of the grouping kernels at max_tokens
   int32_t mt_max;      // upper bound of m-tiles per stage
@@ -60,7 +61,6 @@ struct pcomoe_layer {
   int device;
   int sm_count;
   int group_chunk;                  // tokens per block of the grouping kernels
-  int use_gather4;                  // A operand of the GEMMs fetched by TMA gather4 (else pre-permuted)
   int tc_ok;                        // sizes and dtype allow the tcgen05 path
 };
 

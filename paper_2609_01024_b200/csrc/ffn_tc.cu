@@ -1,16 +1,20 @@
 // K3 / K4: the two grouped GEMMs of the layer on the 5th-generation tensor cores.
 //
-//   K3 (stage 1, expansion side U_e of Sec. 4.1): for every source group, rows gathered from h,
-//       [rows,H] x [W_gate | W_up]^T with SiLU(gate)*up fused in the epilogue -> U (bf16).
+//   K3 (stage 1, expansion side U_e of Sec. 4.1): for every source group, the rows of h of its
+//       (token, source) slots, [rows,H] x [W_gate | W_up]^T with SiLU(gate)*up fused in the epilogue.
+//       The epilogue writes each bf16 row of U straight to the stage-2 position of every path that
+//       reuses it (Sec. 4.3: one U_i(h) per unique source, read by all of its targets), so stage 2
+//       needs no gather.  While the first tile's MMAs run, the epilogue warps also clear y.
 //   K4 (stage 2, projection side D_e and the weighted path sum of Sec. 4.3): for every target
-//       group, rows gathered from U, [rows,F] x W_down^T, scaled by the path weight and added
-//       into y[token] with vector reductions (the scatter-combine back to token order).
+//       group, [rows,F] x W_down^T, scaled by the path weight and added into y[token] with vector
+//       reductions (the scatter-combine back to token order).
+//   The shared expert rides in the same two launches as a second run of tiles (one identity group).
 //
 // One persistent CTA per SM walks a tile list derived on the device by the grouping step
 // (groups padded to 128-row tiles).  Warp roles: warp 0 feeds a 4-stage shared-memory ring with
-// TMA (tile::gather4 row gathers for the A operand, tiled loads for the weights), warp 1 issues
-// tcgen05.mma (128 x 256 x 16, bf16 in, fp32 accumulate in TMEM, two accumulator stages), warps
-// 2-5 drain TMEM with tcgen05.ld and run the epilogue while the next tile's MMAs proceed.
+// TMA tile loads (128-byte swizzle), warp 1 issues tcgen05.mma (128 x 256 x 16, bf16 in, fp32
+// accumulate in TMEM, two accumulator stages), warps 2-5 drain TMEM with tcgen05.ld and run the
+// epilogue while the next tile's MMAs proceed.
 // Every wait on an mbarrier is bounded: on expiry the CTA records PCOMOE_ERR_TIMEOUT, lets its
 // copies land, frees TMEM and returns.
 #include <cuda.h>
@@ -28,24 +32,39 @@ constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t ACC_COLS = 256;                  // fp32 accumulator columns per stage
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int kThreads = 192;
+constexpr int kDstRegs = 8;                 // stage-1 epilogue keeps up to this many destinations in registers
 constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
 
-struct TcParams {
+// One run of tiles that share tensor maps, k-loop length and epilogue parameters: the routed groups, or
+// the shared expert (a single group whose rows are the tokens themselves).
+struct Seg {
   const int32_t *tile_base;    // [G+1] prefix of m-tiles per group (device); NULL: one group
   const int32_t *row_offsets;  // [G+1] unpadded row offsets per group (device); NULL: one group
-  const int32_t *a_idx;        // row gather map of the padded layout; NULL: A row = padded row
   int32_t G;
   int32_t single_rows;         // rows of the single group when tile_base is NULL
   int32_t nt;                  // tiles along N
   int32_t kb;                  // k-blocks
   int32_t b_group_rows;        // rows of the weight tensor per group (0 for a single group)
-  __nv_bfloat16 *u_out;        // stage 1 output (padded rows), leading dimension ldu
+  // stage 1: where a row's SwiGLU output goes
+  const int32_t *row_token;    // token of a padded row (routed), NULL: the row is its own destination
+  const int32_t *path_prow1;   // [T,K] padded stage-1 row of every path
+  const int32_t *path_pos2;    // [T,K] padded stage-2 row of every path (= row of u_out to write)
+  __nv_bfloat16 *u_out;
   int32_t ldu;
-  const int32_t *row_token;    // stage 2: token of an unpadded row; NULL: identity
-  const float *row_w;          // stage 2: weight of an unpadded row; NULL: 1
+  // stage 2: where a row's projection goes
+  const int32_t *s2_token;     // token of an unpadded row; NULL: identity
+  const float *s2_w;           // weight of an unpadded row; NULL: 1
+};
+
+struct TcParams {
+  Seg seg[2];
+  int32_t nseg;
+  int32_t K;
   float *y;
   int32_t ldy;
   int32_t T;
+  float4 *zero_ptr;            // stage 1 only: buffer the epilogue warps clear before their first tile
+  int64_t zero_vec4;           //               (y, so that stage 2 can accumulate into it); 0: nothing
   DevPlan *plan;
 };
 
@@ -99,15 +118,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
-// Four rows (r0..r3) of the 2-D tensor, columns [x, x+64), land as four consecutive 128-byte rows.
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t r0,
-                                            int32_t r1, int32_t r2, int32_t r3, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
-      : "memory");
-}
-
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -169,41 +179,59 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
 }
 
 struct TileInfo {
-  int g, m_idx, n_idx;
+  int seg, g, m_idx, n_idx;
   int prow0;    // first padded row of the tile
   int urow0;    // first unpadded row of the tile
   int valid;    // rows of the tile that exist
 };
 
-// Tiles are numbered group by group; inside a group the m-tiles run fastest so that CTAs working
-// at the same time share one slice of the group's weights.
+// Tiles are numbered segment by segment and group by group; inside a group the m-tiles run fastest so
+// that CTAs working at the same time share one slice of the group's weights.
 struct TileWalker {
-  const int32_t *tb, *ro;
-  int nt, G, g;
-  __device__ TileWalker(const int32_t *tb_, const int32_t *ro_, int nt_, int G_) : tb(tb_), ro(ro_), nt(nt_), G(G_), g(0) {}
-  __device__ int total() const { return tb[G] * nt; }
+  const int32_t *tb, *ro;      // [2][kMaxExperts + 2] each
+  int nt[2], G[2], nseg;
+  int seg, g, seg_first;       // current segment, group, and the first tile id of the segment
+  __device__ int seg_tiles(int s) const { return tb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
+  __device__ int total() const {
+    int t = 0;
+    for (int s = 0; s < nseg; ++s) t += seg_tiles(s);
+    return t;
+  }
   __device__ TileInfo at(int tile) {
-    while (g + 1 < G && tile >= tb[g + 1] * nt) ++g;
+    while (seg + 1 < nseg && tile >= seg_first + seg_tiles(seg)) {
+      seg_first += seg_tiles(seg);
+      ++seg;
+      g = 0;
+    }
+    const int32_t *b = tb + seg * (kMaxExperts + 2), *r = ro + seg * (kMaxExperts + 2);
+    const int n_t = nt[seg], local_seg = tile - seg_first;
+    while (g + 1 < G[seg] && local_seg >= b[g + 1] * n_t) ++g;
     TileInfo t;
-    const int mt = tb[g + 1] - tb[g];
-    const int local = tile - tb[g] * nt;
+    const int mt = b[g + 1] - b[g];
+    const int local = local_seg - b[g] * n_t;
+    t.seg = seg;
     t.g = g;
     t.n_idx = local / mt;
     t.m_idx = local - t.n_idx * mt;
-    t.prow0 = (tb[g] + t.m_idx) * kTileM;
-    t.urow0 = ro[g] + t.m_idx * kTileM;
-    t.valid = min(kTileM, ro[g + 1] - t.urow0);
+    t.prow0 = (b[g] + t.m_idx) * kTileM;
+    t.urow0 = r[g] + t.m_idx * kTileM;
+    t.valid = min(kTileM, r[g + 1] - t.urow0);
     return t;
   }
 };
 
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f + __expf(-g)) * u; }
+
 // STAGE = 1: SwiGLU epilogue (B = 128 gate rows | 128 up rows);  STAGE = 2: weighted scatter-add epilogue.
+// Tensor maps: A, B (gate or down), B2 (up; unused in stage 2) for segment 0 and for segment 1.
 template <int STAGE>
 __global__ void __launch_bounds__(kThreads, 1)
-grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
-                    const __grid_constant__ CUtensorMap tmB1, const TcParams p) {
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                    const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
+                    const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmC1,
+                    const TcParams p) {
   extern __shared__ unsigned char smem_dyn[];
-  __shared__ int32_t s_tb[kMaxExperts + 2], s_ro[kMaxExperts + 2];
+  __shared__ int32_t s_tb[2 * (kMaxExperts + 2)], s_ro[2 * (kMaxExperts + 2)];
   __shared__ __align__(8) uint64_t s_bar[2 * STAGES + 4];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -216,14 +244,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
   auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
 
-  if (p.tile_base) {
-    for (int i = threadIdx.x; i <= p.G; i += blockDim.x) {
-      s_tb[i] = p.tile_base[i];
-      s_ro[i] = p.row_offsets[i];
+  for (int sg = 0; sg < p.nseg; ++sg) {
+    const Seg &S = p.seg[sg];
+    int32_t *tb = s_tb + sg * (kMaxExperts + 2), *ro = s_ro + sg * (kMaxExperts + 2);
+    if (S.tile_base) {
+      for (int i = threadIdx.x; i <= S.G; i += blockDim.x) {
+        tb[i] = S.tile_base[i];
+        ro[i] = S.row_offsets[i];
+      }
+    } else if (threadIdx.x == 0) {
+      tb[0] = 0; tb[1] = (S.single_rows + kTileM - 1) / kTileM;
+      ro[0] = 0; ro[1] = S.single_rows;
     }
-  } else if (threadIdx.x == 0) {
-    s_tb[0] = 0; s_tb[1] = (p.single_rows + kTileM - 1) / kTileM;
-    s_ro[0] = 0; s_ro[1] = p.single_rows;
   }
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -248,43 +280,43 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t tmem_base = s_tmem;
   volatile int *abort_flag = &s_abort;
 
-  const int G = p.tile_base ? p.G : 1;
-  TileWalker walk(s_tb, s_ro, p.nt, G);
+  TileWalker walk;
+  walk.tb = s_tb; walk.ro = s_ro; walk.nseg = p.nseg;
+  for (int sg = 0; sg < 2; ++sg) {
+    walk.nt[sg] = p.seg[sg].nt;
+    walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
+  }
+  walk.seg = 0; walk.g = 0; walk.seg_first = 0;
   const int total = walk.total();
 
   if (warp == 0) {
     // ---------------- producer: TMA into the ring ----------------
-    int stage = 0;
-    uint32_t phase = 0;
-    bool alive = true;
-    for (int tile = blockIdx.x; tile < total && alive; tile += gridDim.x) {
-      const TileInfo t = walk.at(tile);
-      int4 rows = make_int4(0, 0, 0, 0);
-      if (p.a_idx) rows = *reinterpret_cast<const int4 *>(p.a_idx + t.prow0 + 4 * lane);
-      const int a_row0 = p.tile_base ? t.prow0 : t.m_idx * kTileM;
-      const int b_row = t.g * p.b_group_rows + t.n_idx * (STAGE == 1 ? 128 : 256);
-      for (int kb = 0; kb < p.kb; ++kb) {
-        // the give-up decision is taken by the whole warp so that no lane is left at the __syncwarp below
-        if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) { alive = false; break; }
-        const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + A_BYTES;
-        if (lane == 0) mbar_arrive_expect_tx(full_bar(stage), STAGE_BYTES);
-        __syncwarp();
-        if (p.a_idx) {
-          tma_gather4(sa + lane * 512u, &tmA, kb * BK, rows.x, rows.y, rows.z, rows.w, full_bar(stage));
-        } else if (lane == 0) {
-          tma_load_2d(sa, &tmA, kb * BK, a_row0, full_bar(stage));
-        }
-        if (lane == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int tile = blockIdx.x; tile < total && alive; tile += gridDim.x) {
+        const TileInfo t = walk.at(tile);
+        const Seg &S = p.seg[t.seg];
+        const CUtensorMap *mA = t.seg ? &tmA1 : &tmA0, *mB = t.seg ? &tmB1 : &tmB0, *mC = t.seg ? &tmC1 : &tmC0;
+        const int a_row0 = t.prow0;
+        const int b_row = t.g * S.b_group_rows + t.n_idx * (STAGE == 1 ? 128 : 256);
+        for (int kb = 0; kb < S.kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { alive = false; break; }
+          const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_arrive_expect_tx(full_bar(stage), STAGE_BYTES);
+          tma_load_2d(sa, mA, kb * BK, a_row0, full_bar(stage));
           if (STAGE == 1) {
-            tma_load_2d(sb, &tmB0, kb * BK, b_row, full_bar(stage));
-            tma_load_2d(sb + B_BYTES / 2, &tmB1, kb * BK, b_row, full_bar(stage));
+            tma_load_2d(sb, mB, kb * BK, b_row, full_bar(stage));
+            tma_load_2d(sb + B_BYTES / 2, mC, kb * BK, b_row, full_bar(stage));
           } else {
-            tma_load_2d(sb, &tmB0, kb * BK, b_row, full_bar(stage));
+            tma_load_2d(sb, mB, kb * BK, b_row, full_bar(stage));
           }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
@@ -292,10 +324,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t phase = 0, acc_phase = 0;
       bool alive = true;
       for (int tile = blockIdx.x; tile < total && alive; tile += gridDim.x) {
+        const TileInfo t = walk.at(tile);
+        const int nkb = p.seg[t.seg].kb;
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
-        for (int kb = 0; kb < p.kb; ++kb) {
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + A_BYTES;
@@ -316,43 +350,92 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ---------------- epilogue: TMEM -> registers -> global ----------------
     const int quarter = warp & 3;               // the TMEM lanes this warp may read
     const int r = quarter * 32 + lane;          // row of the tile
+    if (STAGE == 1 && p.zero_vec4 > 0) {
+      // clear this CTA's slice of y while the first tile's MMAs are in flight
+      const int et = (warp - 2) * 32 + lane;    // 0..127
+      const int64_t per = (p.zero_vec4 + gridDim.x - 1) / gridDim.x;
+      const int64_t lo = per * blockIdx.x, hi = min(p.zero_vec4, lo + per);
+      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int64_t i = lo + et; i < hi; i += 128) p.zero_ptr[i] = z;
+    }
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       const TileInfo t = walk.at(tile);
+      const Seg &S = p.seg[t.seg];
+      const bool valid = r < t.valid;
+      // destinations are looked up before the wait so the loads overlap the MMAs
+      int token = 0;
+      float wgt = 0.0f;
+      int my_prow = t.prow0 + r;
+      if (STAGE == 1) {
+        if (valid && S.row_token) token = S.row_token[my_prow];
+      } else if (valid) {
+        const int urow = t.urow0 + r;
+        token = S.s2_token ? S.s2_token[urow] : urow;
+        wgt = S.s2_w ? S.s2_w[urow] : 1.0f;
+      }
+      bool ok = valid && (unsigned)token < (unsigned)p.T;
+      if (valid && !ok) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
+      // stage 1, routed rows: the stage-2 rows this (token, source) slot feeds, one per path that reuses it
+      int dst[kDstRegs];
+      int nd = 0;
+      const bool dst_in_regs = p.K <= kDstRegs;
+      if (STAGE == 1 && ok && S.row_token && dst_in_regs) {
+#pragma unroll
+        for (int k = 0; k < kDstRegs; ++k) {
+          if (k < p.K && S.path_prow1[(size_t)token * p.K + k] == my_prow) {
+            const int d = S.path_pos2[(size_t)token * p.K + k];
+#pragma unroll
+            for (int j = 0; j < kDstRegs; ++j)
+              if (j == nd) dst[j] = d;
+            ++nd;
+          }
+        }
+      }
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
       if (STAGE == 1) {
-        const int out_row = (p.tile_base ? t.prow0 : t.m_idx * kTileM) + r;
-        __nv_bfloat16 *dst = p.u_out + (size_t)out_row * p.ldu + (size_t)t.n_idx * 128;
+        const size_t col0 = (size_t)t.n_idx * 128;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 16) {
           float gv[16], uv[16];
           tmem_ld16x2(taddr + c0, taddr + 128 + c0, gv, uv);
+          if (!ok) continue;
           uint32_t packed[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float a0 = gv[2 * i] / (1.0f + __expf(-gv[2 * i])) * uv[2 * i];
-            const float a1 = gv[2 * i + 1] / (1.0f + __expf(-gv[2 * i + 1])) * uv[2 * i + 1];
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(silu_mul(gv[2 * i], uv[2 * i]), silu_mul(gv[2 * i + 1], uv[2 * i + 1]));
             packed[i] = *reinterpret_cast<uint32_t *>(&h2);
           }
-          uint4 *d4 = reinterpret_cast<uint4 *>(dst + c0);
-          d4[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          d4[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+          const uint4 lo = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          const uint4 hi = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+          if (S.row_token && dst_in_regs) {
+#pragma unroll
+            for (int j = 0; j < kDstRegs; ++j) {
+              if (j < nd) {
+                uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)dst[j] * S.ldu + col0 + c0);
+                d4[0] = lo;
+                d4[1] = hi;
+              }
+            }
+          } else if (S.row_token) {
+            // more paths per token than destination registers: look the copies up again per chunk
+            for (int k = 0; k < p.K; ++k) {
+              if (S.path_prow1[(size_t)token * p.K + k] != my_prow) continue;
+              const int dst_row = S.path_pos2[(size_t)token * p.K + k];
+              uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)dst_row * S.ldu + col0 + c0);
+              d4[0] = lo;
+              d4[1] = hi;
+            }
+          } else {
+            uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)my_prow * S.ldu + col0 + c0);
+            d4[0] = lo;
+            d4[1] = hi;
+          }
         }
       } else {
-        const bool valid = r < t.valid;
-        const int urow = t.urow0 + r;
-        int token = 0;
-        float wgt = 0.0f;
-        if (valid) {
-          token = p.row_token ? p.row_token[urow] : urow;
-          wgt = p.row_w ? p.row_w[urow] : 1.0f;
-        }
-        const bool ok = valid && (unsigned)token < (unsigned)p.T;
-        if (valid && !ok) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
         float *dst = p.y + (size_t)token * p.ldy + (size_t)t.n_idx * 256;
 #pragma unroll 1
         for (int c0 = 0; c0 < 256; c0 += 16) {
@@ -446,10 +529,13 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   const int32_t *tb1 = reinterpret_cast<const int32_t *>(ws + lay.tile_base1);
   const int32_t *tb2 = reinterpret_cast<const int32_t *>(ws + lay.tile_base2);
   const int32_t *a1 = reinterpret_cast<const int32_t *>(ws + lay.a1_idx);
-  const int32_t *a2 = reinterpret_cast<const int32_t *>(ws + lay.a2_idx);
-  __nv_bfloat16 *U = reinterpret_cast<__nv_bfloat16 *>(ws + lay.u);
+  const int32_t *prow1 = reinterpret_cast<const int32_t *>(ws + lay.path_prow1);
+  const int32_t *pos2 = reinterpret_cast<const int32_t *>(ws + lay.path_pos2);
+  __nv_bfloat16 *U = reinterpret_cast<__nv_bfloat16 *>(ws + lay.u);        // padded stage-2 order
   __nv_bfloat16 *Ush = reinterpret_cast<__nv_bfloat16 *>(ws + lay.u_sh);
+  uint4 *Hg = reinterpret_cast<uint4 *>(ws + lay.h_gath);                   // padded stage-1 order
   const size_t pad_rows = (size_t)lay.mt_max * kTileM;
+  if (Fsh == 0) stages &= ~(kStage1Shared | kStage2Shared);
 
   static bool attr_done = false;
   if (!attr_done) {
@@ -457,76 +543,67 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     attr_done = true;
   }
-
-  CUtensorMap mA1, mG, mU, mA2, mD;
-  bool ok = true;
-  const void *a1_src = h;
-  const void *a2_src = U;
-  if (!L->use_gather4) {
-    // gather-free fallback: rows are first copied into the padded order, then loaded as plain tiles
-    uint4 *p1 = reinterpret_cast<uint4 *>(ws + lay.a_perm1);
-    if (stages & kStage1Routed) {
-      gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(p1, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
-      count_launch();
-    }
-    a1_src = p1;
-    a2_src = ws + lay.a_perm2;
-    ok = ok && make_map(&mA1, a1_src, pad_rows, H, kTileM);
-    ok = ok && make_map(&mA2, a2_src, pad_rows, F, kTileM);
-  } else {
-    ok = ok && make_map(&mA1, h, (uint64_t)T, H, 1);
-    ok = ok && make_map(&mA2, U, pad_rows, F, 1);
-  }
-  ok = ok && make_map(&mG, wg, (uint64_t)n * F, H, 128);
-  ok = ok && make_map(&mU, wu, (uint64_t)n * F, H, 128);
-  ok = ok && make_map(&mD, wd, (uint64_t)n * H, F, 256);
-  if (!ok) return PCOMOE_ERR_CUDA;
-
   const int grid = L->sm_count;
-  TcParams p1{};
-  p1.tile_base = tb1; p1.row_offsets = g->s1_offsets; p1.a_idx = L->use_gather4 ? a1 : nullptr;
-  p1.G = n; p1.nt = F / 128; p1.kb = H / BK; p1.b_group_rows = F;
-  p1.u_out = U; p1.ldu = F; p1.T = T; p1.plan = plan;
-  if (stages & kStage1Routed) {
-    grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA1, mG, mU, p1);
-    count_launch();
-  }
 
-  CUtensorMap mHs, mSg, mSu, mUs, mSd;
-  if (Fsh > 0) {
-    ok = make_map(&mHs, h, (uint64_t)T, H, kTileM) && make_map(&mSg, sg, Fsh, H, 128) &&
-         make_map(&mSu, su, Fsh, H, 128) && make_map(&mUs, Ush, (uint64_t)lay.t_pad, Fsh, kTileM) &&
-         make_map(&mSd, sd, H, Fsh, 256);
-    if (!ok) return PCOMOE_ERR_CUDA;
-    TcParams s1{};
-    s1.G = 1; s1.single_rows = T; s1.nt = Fsh / 128; s1.kb = H / BK; s1.b_group_rows = 0;
-    s1.u_out = Ush; s1.ldu = Fsh; s1.T = T; s1.plan = plan;
-    if (stages & kStage1Shared) {
-      grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mHs, mSg, mSu, s1);
+  // ---- stage 1: rows of h gathered into group order, then one launch over routed + shared tiles ----
+  if (stages & (kStage1Routed | kStage1Shared)) {
+    CUtensorMap mA[2], mB[2], mC[2];
+    TcParams p{};
+    p.K = c.top_k; p.T = T; p.plan = plan; p.y = y; p.ldy = H;
+    int ns = 0;
+    bool ok = true;
+    if (stages & kStage1Routed) {
+      gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(Hg, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
       count_launch();
+      ok = ok && make_map(&mA[ns], Hg, pad_rows, H, kTileM) && make_map(&mB[ns], wg, (uint64_t)n * F, H, 128) &&
+           make_map(&mC[ns], wu, (uint64_t)n * F, H, 128);
+      Seg &S = p.seg[ns++];
+      S.tile_base = tb1; S.row_offsets = g->s1_offsets; S.G = n; S.nt = F / 128; S.kb = H / BK; S.b_group_rows = F;
+      S.row_token = a1; S.path_prow1 = prow1; S.path_pos2 = pos2; S.u_out = U; S.ldu = F;
     }
-  }
-
-  if (!L->use_gather4 && (stages & kStage2Routed)) {
-    uint4 *p2 = reinterpret_cast<uint4 *>(ws + lay.a_perm2);
-    gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(p2, reinterpret_cast<const uint4 *>(U), a2, tb2, n, F / 8);
+    if (stages & kStage1Shared) {
+      ok = ok && make_map(&mA[ns], h, (uint64_t)T, H, kTileM) && make_map(&mB[ns], sg, Fsh, H, 128) &&
+           make_map(&mC[ns], su, Fsh, H, 128);
+      Seg &S = p.seg[ns++];
+      S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
+    }
+    if (!ok) return PCOMOE_ERR_CUDA;
+    if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; mC[1] = mC[0]; }
+    p.nseg = ns;
+    if (stages & kStage2Routed) {   // a full forward: y is cleared here, under the first tile's MMAs
+      p.zero_ptr = reinterpret_cast<float4 *>(y);
+      p.zero_vec4 = (int64_t)T * H / 4;
+    }
+    grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p);
     count_launch();
   }
-  TcParams p2{};
-  p2.tile_base = tb2; p2.row_offsets = g->s2_offsets; p2.a_idx = L->use_gather4 ? a2 : nullptr;
-  p2.G = n; p2.nt = H / 256; p2.kb = F / BK; p2.b_group_rows = H;
-  p2.row_token = g->s2_token; p2.row_w = g->s2_w; p2.y = y; p2.ldy = H; p2.T = T; p2.plan = plan;
-  if (stages & kStage2Routed) {
-    PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * H, st));
-    grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA2, mD, mD, p2);
-    count_launch(2);
-  }
 
-  if (Fsh > 0 && (stages & kStage2Shared)) {
-    TcParams s2{};
-    s2.G = 1; s2.single_rows = T; s2.nt = H / 256; s2.kb = Fsh / BK; s2.b_group_rows = 0;
-    s2.y = y; s2.ldy = H; s2.T = T; s2.plan = plan;
-    grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mUs, mSd, mSd, s2);
+  // ---- stage 2: one launch over routed + shared tiles, accumulating into y ----
+  if (stages & (kStage2Routed | kStage2Shared)) {
+    CUtensorMap mA[2], mB[2];
+    TcParams p{};
+    p.K = c.top_k; p.T = T; p.plan = plan; p.y = y; p.ldy = H;
+    int ns = 0;
+    bool ok = true;
+    if (stages & kStage2Routed) {
+      if (!(stages & (kStage1Routed | kStage1Shared))) {   // stage 2 on its own: clear y first
+        PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * H, st));
+        count_launch();
+      }
+      ok = ok && make_map(&mA[ns], U, pad_rows, F, kTileM) && make_map(&mB[ns], wd, (uint64_t)n * H, F, 256);
+      Seg &S = p.seg[ns++];
+      S.tile_base = tb2; S.row_offsets = g->s2_offsets; S.G = n; S.nt = H / 256; S.kb = F / BK; S.b_group_rows = H;
+      S.s2_token = g->s2_token; S.s2_w = g->s2_w;
+    }
+    if (stages & kStage2Shared) {
+      ok = ok && make_map(&mA[ns], Ush, (uint64_t)lay.t_pad, Fsh, kTileM) && make_map(&mB[ns], sd, H, Fsh, 256);
+      Seg &S = p.seg[ns++];
+      S.G = 1; S.single_rows = T; S.nt = H / 256; S.kb = Fsh / BK; S.b_group_rows = 0;
+    }
+    if (!ok) return PCOMOE_ERR_CUDA;
+    if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; }
+    p.nseg = ns;
+    grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p);
     count_launch();
   }
   PCOMOE_CUDA_TRY(cudaGetLastError());

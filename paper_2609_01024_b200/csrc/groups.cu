@@ -21,7 +21,8 @@ struct GroupParams {
   DevPlan *plan;
   int32_t *tile_base1, *tile_base2;   // [n+1]
   int32_t *blk_cnt;                   // [NB][2][n]
-  int32_t *a1_idx, *a2_idx;
+  int32_t *a1_idx;                    // token of every padded stage-1 row
+  int32_t *path_prow1, *path_pos2;    // [T,K] padded stage-1 / stage-2 row of every path
   int32_t T, n, K, dedup, chunk, nb;
 };
 
@@ -111,6 +112,8 @@ __global__ void __launch_bounds__(1024) group_scan_kernel(const GroupParams p) {
       if (e < p.n) {
         offs[e] = carry_rows + ir - c;
         tb[e] = carry_tiles + it - tl;
+        if (warp == 0)  // the padding rows of a source group gather token 0 (any valid row will do)
+          for (int x = c; x < tl * kTileM; ++x) p.a1_idx[(size_t)(carry_tiles + it - tl) * kTileM + x] = 0;
       }
       empty += __popc(__ballot_sync(0xffffffffu, e < p.n && c == 0));
       carry_rows += __shfl_sync(0xffffffffu, ir, 31);
@@ -193,7 +196,11 @@ __global__ void group_scatter_kernel(const GroupParams p) {
   }
   for (int k = 0; k < p.K; ++k) {
     const int j = rt[k];
-    if (j < 0) continue;
+    if (j < 0) {  // a path with an out-of-range expert id feeds no row
+      p.path_prow1[(size_t)t * p.K + k] = -1;
+      p.path_pos2[(size_t)t * p.K + k] = -1;
+      continue;
+    }
     const int idx = tl * p.K + k;
     const int r2 = off2[j] + bo2[j] + bits_below(bits2 + (size_t)j * W, idx);
     const int q = t * p.K + k;
@@ -202,7 +209,8 @@ __global__ void group_scatter_kernel(const GroupParams p) {
     p.g.s2_s1row[r2] = myrow[k];
     p.g.s2_token[r2] = t;
     p.g.s2_w[r2] = p.w[q];
-    p.a2_idx[(size_t)tb2[j] * kTileM + (r2 - off2[j])] = tb1[s] * kTileM + (myrow[k] - off1[s]);
+    p.path_prow1[q] = tb1[s] * kTileM + (myrow[k] - off1[s]);
+    p.path_pos2[q] = tb2[j] * kTileM + (r2 - off2[j]);
   }
 }
 
@@ -217,14 +225,14 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
   p.tile_base2 = reinterpret_cast<int32_t *>(ws + lay.tile_base2);
   p.blk_cnt = reinterpret_cast<int32_t *>(ws + lay.blk_cnt);
   p.a1_idx = reinterpret_cast<int32_t *>(ws + lay.a1_idx);
-  p.a2_idx = reinterpret_cast<int32_t *>(ws + lay.a2_idx);
+  p.path_prow1 = reinterpret_cast<int32_t *>(ws + lay.path_prow1);
+  p.path_pos2 = reinterpret_cast<int32_t *>(ws + lay.path_pos2);
   p.T = T; p.n = c.n_experts; p.K = c.top_k; p.dedup = c.dedup; p.chunk = L->group_chunk;
   p.nb = (T + p.chunk - 1) / p.chunk;
 
-  // status word, plan, and the padding entries of the gather maps start from zero
+  // the status word and the plan start from zero (the scan kernel fills the padding of the gather map)
   PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.plan, 0, sizeof(DevPlan), st));
-  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.a1_idx, 0, lay.u - lay.a1_idx, st));
-  count_launch(2);
+  count_launch();
 
   const int CK = p.chunk * p.K, W = (CK + 31) / 32;
   const size_t smem_count = sizeof(int32_t) * ((size_t)2 * CK + 2 * p.n);

@@ -59,6 +59,7 @@ extern "C" pcomoe_status pcomoe_build_path_groups_static(const pcomoe_layer *L, 
   char *scratch = nullptr;
   const pcomoe_status s = scratch_for_current_device(dev, &scratch);
   if (s != PCOMOE_OK) return s;
-  // launch_groups zero-fills the header and the gather maps itself, so nothing of an earlier call survives
+  // launch_groups zero-fills the header and rewrites every entry it later reads, so nothing of an earlier
+  // call survives
   return launch_groups(L, T, d_path_src, d_path_tgt, d_path_w, out, scratch, lay, (cudaStream_t)stream);
 }

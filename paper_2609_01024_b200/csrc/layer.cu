@@ -35,13 +35,11 @@ WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
   w.tile_base2 = take(sizeof(int32_t) * (c.n_experts + 1));
   w.blk_cnt = take(sizeof(int32_t) * (size_t)w.nb_max * 2 * c.n_experts);
   w.a1_idx = take(sizeof(int32_t) * (size_t)w.mt_max * kTileM);
-  w.a2_idx = take(sizeof(int32_t) * (size_t)w.mt_max * kTileM);
+  w.path_prow1 = take(sizeof(int32_t) * (size_t)Pm);
+  w.path_pos2 = take(sizeof(int32_t) * (size_t)Pm);
   w.u = take(es * (size_t)w.mt_max * kTileM * c.ffn);
   w.u_sh = take(es * (size_t)w.t_pad * c.shared_ffn);
-  if (L->tc_ok && !L->use_gather4) {
-    w.a_perm1 = take(es * (size_t)w.mt_max * kTileM * c.hidden);
-    w.a_perm2 = take(es * (size_t)w.mt_max * kTileM * c.ffn);
-  }
+  if (L->tc_ok) w.h_gath = take(es * (size_t)w.mt_max * kTileM * c.hidden);
   w.total = off;
   return w;
 }
@@ -76,8 +74,6 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
     delete L;
     return PCOMOE_ERR_UNSUPPORTED;
   }
-  const char *g4 = std::getenv("PCOMOE_GATHER4");
-  L->use_gather4 = g4 ? (std::atoi(g4) != 0) : 0;
 
   int cnt = 0;
   for (int i = 0; i < n * n; ++i) cnt += h_mask[i] ? 1 : 0;

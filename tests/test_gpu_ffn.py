@@ -49,7 +49,8 @@ TC_SHAPES = [dict(T=70, H=256, F=128, n=5, K=2),                                
              dict(T=1500, H=1024, F=1408, n=8, K=2),                                       # several tiles + tail
              dict(T=257, H=256, F=256, n=60, K=4, F_sh=512, mask_p=0.3, logits="zipf", zipf_a=1.2),  # empty groups
              dict(T=1, H=256, F=128, n=4, K=2),
-             dict(T=129, H=256, F=128, n=3, K=3, mask_p=1.0)]                              # K = n, heavy reuse
+             dict(T=129, H=256, F=128, n=3, K=3, mask_p=1.0),                              # K = n, heavy reuse
+             dict(T=100, H=256, F=128, n=16, K=12, mask_p=0.5)]                            # K beyond the register path
 
 
 @pytest.mark.parametrize("dedup", [1, 0])
