@@ -164,6 +164,8 @@ def main():
                     help="only run warm-up + steps of the device-resident hot path, print a short line and exit")
     ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ffn-impl", type=int, default=0,
+                    help="pcomoe_ffn_impl: 0 auto, 1 SIMT, 2 tcgen05 one CTA per tile, 3 tcgen05 CTA pairs")
     ap.add_argument("--variant", default="default", choices=["default", "vanilla"],
                     help="vanilla: diagonal-only mask (every path a whole expert, no reuse)")
     args = ap.parse_args()
@@ -205,7 +207,7 @@ def main():
                            w_gate=B.to_device(L.w_gate, dev), w_up=B.to_device(L.w_up, dev),
                            w_down=B.to_device(L.w_down, dev),
                            shared=tuple(B.to_device(x, dev) for x in (L.wsh_gate, L.wsh_up, L.wsh_down)) if cfg.F_sh else None,
-                           max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam, device=dev)
+                           max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam, ffn_impl=args.ffn_impl, device=dev)
     d_logits = torch.from_numpy(L.logits).to(dev)
     d_h = B.to_device(L.h, dev)
     stream = torch.cuda.current_stream()

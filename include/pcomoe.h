@@ -46,10 +46,13 @@ typedef enum { PCOMOE_BF16 = 0, PCOMOE_FP32 = 1 } pcomoe_dtype;
 
 /* Which kernels pcomoe_ffn_forward uses. */
 typedef enum {
-  PCOMOE_FFN_AUTO = 0,   /* tensor-core path when dtype and sizes allow, else the SIMT path */
+  PCOMOE_FFN_AUTO = 0,   /* tensor-core path when dtype and sizes allow (CTA pairs when groups average
+                            at least 256 rows, else one CTA per tile), else the SIMT path        */
   PCOMOE_FFN_SIMT = 1,   /* plain-FMA kernels (any size, bf16 or fp32 storage)               */
-  PCOMOE_FFN_TCGEN05 = 2 /* tcgen05 / TMEM / TMA kernels; PCOMOE_ERR_UNSUPPORTED if not bf16
-                            or if H % 256 != 0 or F % 128 != 0                               */
+  PCOMOE_FFN_TCGEN05 = 2, /* tcgen05 / TMEM / TMA kernels, one CTA per 128 x 256 tile;
+                             PCOMOE_ERR_UNSUPPORTED if not bf16 or if H % 256 != 0 or F % 128 != 0 */
+  PCOMOE_FFN_TCGEN05_PAIR = 3 /* the same with two CTAs (a cluster of 2 SMs) per 256 x 256 tile,
+                                 tcgen05.mma.cta_group::2; same size rules                        */
 } pcomoe_ffn_impl;
 
 /* Plain data; set struct_size = sizeof(pcomoe_config). */

@@ -80,14 +80,17 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One probe of the barrier.  The thread may sleep in hardware for up to `kSuspendNs` until the phase
+// completes, so a waiting warp issues a handful of instructions instead of spinning.
+constexpr uint32_t kSuspendNs = 200000u;
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendNs)
       : "memory");
   return ok;
 }
@@ -100,12 +103,10 @@ __device__ __forceinline__ uint64_t global_ns() {
 __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
-  for (uint32_t it = 1; it < (1u << 30); ++it) {
+  for (uint32_t it = 1; it < (1u << 24); ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) break;
-    }
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   return false;
@@ -141,37 +142,24 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 16 accumulator columns of this thread's TMEM lane, and the wait for them, in one statement
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
-  uint32_t r[16];
+// 32 accumulator columns of this thread's TMEM lane.  The load is asynchronous: tmem_wait_ld() must come
+// before the registers are read, and reg_fence32() ties their first use to a point after that wait.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-// the same for two column ranges at once (gate and up halves of a stage-1 accumulator)
-__device__ __forceinline__ void tmem_ld16x2(uint32_t ta, uint32_t tb, float *a, float *b) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%32];\n\t"
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(ta), "r"(tb)
+      : "r"(taddr)
       : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void reg_fence32(uint32_t (&r)[32]) {
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    a[i] = __uint_as_float(r[i]);
-    b[i] = __uint_as_float(r[16 + i]);
-  }
+  for (int i = 0; i < 32; ++i) asm volatile("" : "+r"(r[i]));
 }
 
 __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d) {
@@ -220,7 +208,142 @@ struct TileWalker {
   }
 };
 
-__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.0f + __expf(-g)) * u; }
+// What an epilogue thread needs to know about its row, looked up before the accumulator is ready so that
+// the loads overlap the MMAs.
+struct RowCtx {
+  bool ok;            // the row exists and its token is in range
+  int token;
+  float wgt;          // stage 2: path weight
+  int my_prow;        // padded row of this thread
+  int nd;             // stage 1, routed: number of stage-2 rows fed by this (token, source) slot
+  int dst[kDstRegs];  //                  and those rows (when K <= kDstRegs)
+  bool dst_in_regs;
+};
+
+template <int STAGE>
+__device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, const TileInfo &t, int r) {
+  RowCtx c;
+  const bool valid = r < t.valid;
+  c.token = 0;
+  c.wgt = 0.0f;
+  c.my_prow = t.prow0 + r;
+  c.nd = 0;
+  c.dst_in_regs = p.K <= kDstRegs;
+  if (STAGE == 1) {
+    if (valid && S.row_token) c.token = S.row_token[c.my_prow];
+  } else if (valid) {
+    const int urow = t.urow0 + r;
+    c.token = S.s2_token ? S.s2_token[urow] : urow;
+    c.wgt = S.s2_w ? S.s2_w[urow] : 1.0f;
+  }
+  c.ok = valid && (unsigned)c.token < (unsigned)p.T;
+  if (valid && !c.ok) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
+  if (STAGE == 1 && c.ok && S.row_token && c.dst_in_regs) {
+#pragma unroll
+    for (int k = 0; k < kDstRegs; ++k) {
+      if (k < p.K && S.path_prow1[(size_t)c.token * p.K + k] == c.my_prow) {
+        const int d = S.path_pos2[(size_t)c.token * p.K + k];
+#pragma unroll
+        for (int j = 0; j < kDstRegs; ++j)
+          if (j == c.nd) c.dst[j] = d;
+        ++c.nd;
+      }
+    }
+  }
+  return c;
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
+// Stage 1: SiLU(gate) * up for 32 columns held in registers, packed to bf16 and written to every
+// stage-2 row that reads this slot (or to the row itself for the shared expert).
+__device__ __forceinline__ void store_swiglu32(const TcParams &p, const Seg &S, const RowCtx &c, size_t col,
+                                               const uint32_t (&g)[32], const uint32_t (&u)[32]) {
+  uint4 out[4];
+  uint32_t *o = reinterpret_cast<uint32_t *>(out);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i])),
+                                              silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
+    o[i] = *reinterpret_cast<uint32_t *>(&h2);
+  }
+  if (S.row_token && c.dst_in_regs) {
+#pragma unroll
+    for (int j = 0; j < kDstRegs; ++j) {
+      if (j < c.nd) {
+        uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)c.dst[j] * S.ldu + col);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) d4[q] = out[q];
+      }
+    }
+  } else if (S.row_token) {
+    // more paths per token than destination registers: look the copies up again
+    for (int k = 0; k < p.K; ++k) {
+      if (S.path_prow1[(size_t)c.token * p.K + k] != c.my_prow) continue;
+      uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)S.path_pos2[(size_t)c.token * p.K + k] * S.ldu + col);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) d4[q] = out[q];
+    }
+  } else {
+    uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)c.my_prow * S.ldu + col);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) d4[q] = out[q];
+  }
+}
+
+// Drains one accumulator (this thread's TMEM lane) and applies the stage's epilogue.  TMEM loads are issued
+// one step ahead of the arithmetic: a tcgen05.ld queues behind the MMAs already issued, so its latency is
+// long while the next tile is being computed, and must overlap the math and the stores of the previous step.
+template <int STAGE>
+__device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, const TileInfo &t, const RowCtx &c,
+                                              uint32_t taddr) {
+  if (STAGE == 1) {
+    const size_t col0 = (size_t)t.n_idx * 128;
+    uint32_t g0[32], u0[32], g1[32], u1[32];
+    tmem_ld32_issue(taddr, g0);
+    tmem_ld32_issue(taddr + 128, u0);
+#pragma unroll
+    for (int c0 = 0; c0 < 128; c0 += 64) {
+      tmem_wait_ld();
+      reg_fence32(g0); reg_fence32(u0);
+      tmem_ld32_issue(taddr + c0 + 32, g1);
+      tmem_ld32_issue(taddr + 128 + c0 + 32, u1);
+      if (c.ok) store_swiglu32(p, S, c, col0 + c0, g0, u0);
+      tmem_wait_ld();
+      reg_fence32(g1); reg_fence32(u1);
+      if (c0 + 64 < 128) {
+        tmem_ld32_issue(taddr + c0 + 64, g0);
+        tmem_ld32_issue(taddr + 128 + c0 + 64, u0);
+      }
+      if (c.ok) store_swiglu32(p, S, c, col0 + c0 + 32, g1, u1);
+    }
+  } else {
+    float *dst = p.y + (size_t)c.token * p.ldy + (size_t)t.n_idx * 256;
+    uint32_t v0[32], v1[32];
+    tmem_ld32_issue(taddr, v0);
+#pragma unroll 1
+    for (int c0 = 0; c0 < 256; c0 += 64) {
+      tmem_wait_ld();
+      reg_fence32(v0);
+      tmem_ld32_issue(taddr + c0 + 32, v1);
+      if (c.ok) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          red_add_v4(dst + c0 + i, c.wgt * __uint_as_float(v0[i]), c.wgt * __uint_as_float(v0[i + 1]),
+                     c.wgt * __uint_as_float(v0[i + 2]), c.wgt * __uint_as_float(v0[i + 3]));
+      }
+      tmem_wait_ld();
+      reg_fence32(v1);
+      if (c0 + 64 < 256) tmem_ld32_issue(taddr + c0 + 64, v0);
+      if (c.ok) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          red_add_v4(dst + c0 + 32 + i, c.wgt * __uint_as_float(v1[i]), c.wgt * __uint_as_float(v1[i + 1]),
+                     c.wgt * __uint_as_float(v1[i + 2]), c.wgt * __uint_as_float(v1[i + 3]));
+      }
+    }
+  }
+}
 
 // STAGE = 1: SwiGLU epilogue (B = 128 gate rows | 128 up rows);  STAGE = 2: weighted scatter-add epilogue.
 // Tensor maps: A, B (gate or down), B2 (up; unused in stage 2) for segment 0 and for segment 1.
@@ -363,91 +486,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       const TileInfo t = walk.at(tile);
       const Seg &S = p.seg[t.seg];
-      const bool valid = r < t.valid;
-      // destinations are looked up before the wait so the loads overlap the MMAs
-      int token = 0;
-      float wgt = 0.0f;
-      int my_prow = t.prow0 + r;
-      if (STAGE == 1) {
-        if (valid && S.row_token) token = S.row_token[my_prow];
-      } else if (valid) {
-        const int urow = t.urow0 + r;
-        token = S.s2_token ? S.s2_token[urow] : urow;
-        wgt = S.s2_w ? S.s2_w[urow] : 1.0f;
-      }
-      bool ok = valid && (unsigned)token < (unsigned)p.T;
-      if (valid && !ok) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
-      // stage 1, routed rows: the stage-2 rows this (token, source) slot feeds, one per path that reuses it
-      int dst[kDstRegs];
-      int nd = 0;
-      const bool dst_in_regs = p.K <= kDstRegs;
-      if (STAGE == 1 && ok && S.row_token && dst_in_regs) {
-#pragma unroll
-        for (int k = 0; k < kDstRegs; ++k) {
-          if (k < p.K && S.path_prow1[(size_t)token * p.K + k] == my_prow) {
-            const int d = S.path_pos2[(size_t)token * p.K + k];
-#pragma unroll
-            for (int j = 0; j < kDstRegs; ++j)
-              if (j == nd) dst[j] = d;
-            ++nd;
-          }
-        }
-      }
+      const RowCtx c = prepare_row<STAGE>(p, S, t, r);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
-      if (STAGE == 1) {
-        const size_t col0 = (size_t)t.n_idx * 128;
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 16) {
-          float gv[16], uv[16];
-          tmem_ld16x2(taddr + c0, taddr + 128 + c0, gv, uv);
-          if (!ok) continue;
-          uint32_t packed[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(silu_mul(gv[2 * i], uv[2 * i]), silu_mul(gv[2 * i + 1], uv[2 * i + 1]));
-            packed[i] = *reinterpret_cast<uint32_t *>(&h2);
-          }
-          const uint4 lo = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          const uint4 hi = make_uint4(packed[4], packed[5], packed[6], packed[7]);
-          if (S.row_token && dst_in_regs) {
-#pragma unroll
-            for (int j = 0; j < kDstRegs; ++j) {
-              if (j < nd) {
-                uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)dst[j] * S.ldu + col0 + c0);
-                d4[0] = lo;
-                d4[1] = hi;
-              }
-            }
-          } else if (S.row_token) {
-            // more paths per token than destination registers: look the copies up again per chunk
-            for (int k = 0; k < p.K; ++k) {
-              if (S.path_prow1[(size_t)token * p.K + k] != my_prow) continue;
-              const int dst_row = S.path_pos2[(size_t)token * p.K + k];
-              uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)dst_row * S.ldu + col0 + c0);
-              d4[0] = lo;
-              d4[1] = hi;
-            }
-          } else {
-            uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)my_prow * S.ldu + col0 + c0);
-            d4[0] = lo;
-            d4[1] = hi;
-          }
-        }
-      } else {
-        float *dst = p.y + (size_t)token * p.ldy + (size_t)t.n_idx * 256;
-#pragma unroll 1
-        for (int c0 = 0; c0 < 256; c0 += 16) {
-          float v[16];
-          tmem_ld16(taddr + c0, v);
-          if (ok) {
-#pragma unroll
-            for (int i = 0; i < 16; i += 4)
-              red_add_v4(dst + c0 + i, wgt * v[i], wgt * v[i + 1], wgt * v[i + 2], wgt * v[i + 3]);
-          }
-        }
-      }
+      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16));
       tc_fence_before();
       mbar_arrive(acce_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -468,6 +510,280 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// =====================================================================================================
+// CTA-pair variant: two CTAs of a cluster (two SMs) share one 256 x 256 tile.  Each CTA stages its own 128
+// rows of A and its own 128-row half of B (the leader: gate rows / first half of W_down; the peer: up rows /
+// second half), so a pair moves 64 KB per k-block where two independent CTAs would move 96 KB, and each
+// SM's shared memory serves half the operand reads.  One thread of the leader issues
+// tcgen05.mma.cta_group::2 (M = 256: rows 0-127 accumulate in the leader's TMEM, rows 128-255 in the
+// peer's); completion is broadcast to both CTAs' barriers with tcgen05.commit ... multicast::cluster.
+// Both CTAs' TMA loads report their bytes to the leader's "full" barrier; both CTAs' epilogues release
+// the leader's "accumulator empty" barrier.  A group with an odd number of 128-row tiles ends with a pair
+// whose peer half has no rows: it is computed and dropped.
+// =====================================================================================================
+constexpr int STAGES2 = 6;
+constexpr uint32_t HALF_BYTES = kTileM * BK * 2;            // 16 KB: A tile, and one CTA's half of B
+constexpr uint32_t STAGE2_BYTES = 2 * HALF_BYTES;           // per CTA
+constexpr uint32_t kIdescPair = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of `local_addr` in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// tile load whose completion bytes are reported to a barrier that may live in the peer CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y,
+                                                 uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(cluster_bar)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescPair), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3)
+               : "memory");
+}
+
+// Pair tiles are numbered segment by segment, group by group; inside a group the pairs of one n-tile
+// run fastest.  CTA `rank` of the pair owns m-tile 2*pair + rank of the group.
+struct PairWalker {
+  const int32_t *tb, *ro, *pb;   // [2][kMaxExperts + 2] each: m-tile prefix, row offsets, pair prefix
+  int nt[2], G[2], nseg;
+  int seg, g, seg_first;
+  __device__ int seg_tiles(int s) const { return pb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
+  __device__ int total() const {
+    int t = 0;
+    for (int s = 0; s < nseg; ++s) t += seg_tiles(s);
+    return t;
+  }
+  __device__ TileInfo at(int tile, int rank) {
+    while (seg + 1 < nseg && tile >= seg_first + seg_tiles(seg)) {
+      seg_first += seg_tiles(seg);
+      ++seg;
+      g = 0;
+    }
+    const int o = seg * (kMaxExperts + 2);
+    const int32_t *b = tb + o, *r = ro + o, *q = pb + o;
+    const int n_t = nt[seg], local_seg = tile - seg_first;
+    while (g + 1 < G[seg] && local_seg >= q[g + 1] * n_t) ++g;
+    TileInfo t;
+    const int np = q[g + 1] - q[g];
+    const int local = local_seg - q[g] * n_t;
+    t.seg = seg;
+    t.g = g;
+    t.n_idx = local / np;
+    t.m_idx = 2 * (local - t.n_idx * np) + rank;
+    t.prow0 = (b[g] + t.m_idx) * kTileM;
+    t.urow0 = r[g] + t.m_idx * kTileM;
+    t.valid = t.m_idx < b[g + 1] - b[g] ? min(kTileM, r[g + 1] - t.urow0) : 0;
+    return t;
+  }
+};
+
+template <int STAGE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                         const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
+                         const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmC1,
+                         const TcParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ int32_t s_tb[2 * (kMaxExperts + 2)], s_ro[2 * (kMaxExperts + 2)], s_pb[2 * (kMaxExperts + 2)];
+  __shared__ __align__(8) uint64_t s_bar[2 * STAGES2 + 4];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const uint32_t bar0 = smem_u32(s_bar);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES2 + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + 2 + a); };
+
+  for (int sg = 0; sg < p.nseg; ++sg) {
+    const Seg &S = p.seg[sg];
+    int32_t *tb = s_tb + sg * (kMaxExperts + 2), *ro = s_ro + sg * (kMaxExperts + 2);
+    if (S.tile_base) {
+      for (int i = threadIdx.x; i <= S.G; i += blockDim.x) {
+        tb[i] = S.tile_base[i];
+        ro[i] = S.row_offsets[i];
+      }
+    } else if (threadIdx.x == 0) {
+      tb[0] = 0; tb[1] = (S.single_rows + kTileM - 1) / kTileM;
+      ro[0] = 0; ro[1] = S.single_rows;
+    }
+  }
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < STAGES2; ++s) {
+      mbar_init(full_bar(s), 1);      // the leader's expect_tx arrival; bytes come from both CTAs
+      mbar_init(empty_bar(s), 1);     // one commit (broadcast to both CTAs)
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accf_bar(a), 1);      // one commit (broadcast)
+      mbar_init(acce_bar(a), 256);    // the epilogue threads of both CTAs
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 0 && lane < p.nseg) {   // pair prefix per group: ceil(m-tiles / 2)
+    const int sg = lane, o = sg * (kMaxExperts + 2);
+    const int G = p.seg[sg].tile_base ? p.seg[sg].G : 1;
+    int acc = 0;
+    for (int g = 0; g < G; ++g) {
+      s_pb[o + g] = acc;
+      acc += (s_tb[o + g + 1] - s_tb[o + g] + 1) >> 1;
+    }
+    s_pb[o + G] = acc;
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                 // both CTAs' barriers exist before anything is signalled across
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem;
+  volatile int *abort_flag = &s_abort;
+
+  PairWalker walk;
+  walk.tb = s_tb; walk.ro = s_ro; walk.pb = s_pb; walk.nseg = p.nseg;
+  for (int sg = 0; sg < 2; ++sg) {
+    walk.nt[sg] = p.seg[sg].nt;
+    walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
+  }
+  walk.seg = 0; walk.g = 0; walk.seg_first = 0;
+  const int total = walk.total();
+
+  if (warp == 0) {
+    // ---------------- producer (both CTAs): own A rows and own half of B ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int tile = pair_id; tile < total && alive; tile += n_pairs) {
+        const TileInfo t = walk.at(tile, rank);
+        const Seg &S = p.seg[t.seg];
+        const CUtensorMap *mA = t.seg ? &tmA1 : &tmA0;
+        const CUtensorMap *mB;
+        int b_row;
+        if (STAGE == 1) {            // leader: 128 gate rows; peer: the matching 128 up rows
+          mB = rank == 0 ? (t.seg ? &tmB1 : &tmB0) : (t.seg ? &tmC1 : &tmC0);
+          b_row = t.g * S.b_group_rows + t.n_idx * 128;
+        } else {                     // halves of a 256-row slice of W_down
+          mB = t.seg ? &tmB1 : &tmB0;
+          b_row = t.g * S.b_group_rows + t.n_idx * 256 + (int)rank * 128;
+        }
+        for (int kb = 0; kb < S.kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { alive = false; break; }
+          const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
+          const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
+          tma_load_2d_pair(sa, mA, kb * BK, t.prow0, lead_full);
+          tma_load_2d_pair(sb, mB, kb * BK, b_row, lead_full);
+          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader only) ----------------
+    if (lane == 0 && rank == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool alive = true;
+      for (int tile = pair_id; tile < total && alive; tile += n_pairs) {
+        const TileInfo t = walk.at(tile, 0);
+        const int nkb = p.seg[t.seg].kb;
+        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
+          const uint64_t da = umma_desc(sa), db = umma_desc(sb);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)
+            umma_bf16_pair(d_tmem, da + 2u * k, db + 2u * k, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(empty_bar(stage));
+          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
+        umma_commit_pair(accf_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue (both CTAs, own 128 rows) ----------------
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;
+    if (STAGE == 1 && p.zero_vec4 > 0) {
+      const int et = (warp - 2) * 32 + lane;
+      const int64_t per = (p.zero_vec4 + gridDim.x - 1) / gridDim.x;
+      const int64_t lo = per * blockIdx.x, hi = min(p.zero_vec4, lo + per);
+      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int64_t i = lo + et; i < hi; i += 128) p.zero_ptr[i] = z;
+    }
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = pair_id; tile < total; tile += n_pairs) {
+      const TileInfo t = walk.at(tile, rank);
+      const Seg &S = p.seg[t.seg];
+      const RowCtx c = prepare_row<STAGE>(p, S, t, r);
+      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
+      tc_fence_after();
+      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16));
+      tc_fence_before();
+      mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));   // the leader's MMA waits for both halves
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (s_abort) {
+    if (threadIdx.x == 0) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_TIMEOUT);
+    const uint64_t t0 = global_ns();
+    for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
+  }
+  cluster_sync_all();                 // no signal may reach a CTA that has already exited
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -515,6 +831,7 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, ui
 }
 
 constexpr size_t kSmemDyn = (size_t)STAGES * STAGE_BYTES + 1024;
+static_assert((size_t)STAGES2 * STAGE2_BYTES + 1024 == kSmemDyn, "both kernels use the same ring size");
 
 }  // namespace
 
@@ -541,9 +858,15 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   if (!attr_done) {
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     attr_done = true;
   }
-  const int grid = L->sm_count;
+  // CTA pairs pay off once groups are a few tiles long; short groups (decode) leave the peer CTA idle
+  const bool pair = c.ffn_impl == PCOMOE_FFN_TCGEN05_PAIR ||
+                    (c.ffn_impl == PCOMOE_FFN_AUTO && (int64_t)T * c.top_k >= (int64_t)256 * n);
+  const int grid = pair ? (L->sm_count & ~1) : L->sm_count;
+  const uint32_t down_box = pair ? 128 : 256;   // a CTA of a pair loads half of the 256-row slice of W_down
 
   // ---- stage 1: rows of h gathered into group order, then one launch over routed + shared tiles ----
   if (stages & (kStage1Routed | kStage1Shared)) {
@@ -574,7 +897,10 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
       p.zero_ptr = reinterpret_cast<float4 *>(y);
       p.zero_vec4 = (int64_t)T * H / 4;
     }
-    grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p);
+    if (pair)
+      grouped_gemm_pair_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p);
+    else
+      grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p);
     count_launch();
   }
 
@@ -590,20 +916,23 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
         PCOMOE_CUDA_TRY(cudaMemsetAsync(y, 0, sizeof(float) * (size_t)T * H, st));
         count_launch();
       }
-      ok = ok && make_map(&mA[ns], U, pad_rows, F, kTileM) && make_map(&mB[ns], wd, (uint64_t)n * H, F, 256);
+      ok = ok && make_map(&mA[ns], U, pad_rows, F, kTileM) && make_map(&mB[ns], wd, (uint64_t)n * H, F, down_box);
       Seg &S = p.seg[ns++];
       S.tile_base = tb2; S.row_offsets = g->s2_offsets; S.G = n; S.nt = H / 256; S.kb = F / BK; S.b_group_rows = H;
       S.s2_token = g->s2_token; S.s2_w = g->s2_w;
     }
     if (stages & kStage2Shared) {
-      ok = ok && make_map(&mA[ns], Ush, (uint64_t)lay.t_pad, Fsh, kTileM) && make_map(&mB[ns], sd, H, Fsh, 256);
+      ok = ok && make_map(&mA[ns], Ush, (uint64_t)lay.t_pad, Fsh, kTileM) && make_map(&mB[ns], sd, H, Fsh, down_box);
       Seg &S = p.seg[ns++];
       S.G = 1; S.single_rows = T; S.nt = H / 256; S.kb = Fsh / BK; S.b_group_rows = 0;
     }
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; }
     p.nseg = ns;
-    grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p);
+    if (pair)
+      grouped_gemm_pair_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p);
+    else
+      grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p);
     count_launch();
   }
   PCOMOE_CUDA_TRY(cudaGetLastError());

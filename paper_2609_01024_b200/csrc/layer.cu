@@ -56,7 +56,7 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
   if (n <= 0 || K <= 0 || cfg->hidden <= 0 || cfg->ffn <= 0 || cfg->shared_ffn < 0)
     return PCOMOE_ERR_INVALID_ARG;
   if (cfg->in_dtype != PCOMOE_BF16 && cfg->in_dtype != PCOMOE_FP32) return PCOMOE_ERR_INVALID_ARG;
-  if (cfg->ffn_impl < PCOMOE_FFN_AUTO || cfg->ffn_impl > PCOMOE_FFN_TCGEN05)
+  if (cfg->ffn_impl < PCOMOE_FFN_AUTO || cfg->ffn_impl > PCOMOE_FFN_TCGEN05_PAIR)
     return PCOMOE_ERR_INVALID_ARG;
   if (K > n || K > kMaxTopK) return PCOMOE_ERR_SHAPE;
   if (n > kMaxExperts) return PCOMOE_ERR_UNSUPPORTED;
@@ -70,7 +70,7 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
   L->cfg = *cfg;
   L->tc_ok = cfg->in_dtype == PCOMOE_BF16 && cfg->hidden % 256 == 0 && cfg->ffn % 128 == 0 &&
              cfg->shared_ffn % 128 == 0;
-  if (cfg->ffn_impl == PCOMOE_FFN_TCGEN05 && !L->tc_ok) {
+  if (cfg->ffn_impl >= PCOMOE_FFN_TCGEN05 && !L->tc_ok) {
     delete L;
     return PCOMOE_ERR_UNSUPPORTED;
   }
@@ -207,7 +207,7 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *L, int32_t T, const 
   WsLayout lay;
   pcomoe_status s = check_ws(L, T, d_workspace, ws_bytes, &lay);
   if (s != PCOMOE_OK) return s;
-  const bool tc = L->cfg.ffn_impl == PCOMOE_FFN_TCGEN05 ||
+  const bool tc = L->cfg.ffn_impl >= PCOMOE_FFN_TCGEN05 ||
                   (L->cfg.ffn_impl == PCOMOE_FFN_AUTO && L->tc_ok);
   if (tc)
     return launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
