@@ -32,6 +32,7 @@ constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t ACC_COLS = 256;                  // fp32 accumulator columns per stage
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int kThreads = 192;
+constexpr int kEpiStride = 36;               // words per row staged by the epilogue: 16-byte aligned, conflict-free
 constexpr int kDstRegs = 8;                 // stage-1 epilogue keeps up to this many destinations in registers
 constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
 
@@ -228,7 +229,7 @@ __device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, c
   c.wgt = 0.0f;
   c.my_prow = t.prow0 + r;
   c.nd = 0;
-  c.dst_in_regs = p.K <= kDstRegs;
+  c.dst_in_regs = p.K <= kDstRegs || !S.row_token;   // the same for every lane of the warp
   if (STAGE == 1) {
     if (valid && S.row_token) c.token = S.row_token[c.my_prow];
   } else if (valid) {
@@ -238,6 +239,10 @@ __device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, c
   }
   c.ok = valid && (unsigned)c.token < (unsigned)p.T;
   if (valid && !c.ok) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
+  if (STAGE == 1 && c.ok && !S.row_token) {   // shared expert: the row is its own destination
+    c.dst[0] = c.my_prow;
+    c.nd = 1;
+  }
   if (STAGE == 1 && c.ok && S.row_token && c.dst_in_regs) {
 #pragma unroll
     for (int k = 0; k < kDstRegs; ++k) {
@@ -255,11 +260,8 @@ __device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, c
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
 
-// Stage 1: SiLU(gate) * up for 32 columns held in registers, packed to bf16 and written to every
-// stage-2 row that reads this slot (or to the row itself for the shared expert).
-__device__ __forceinline__ void store_swiglu32(const TcParams &p, const Seg &S, const RowCtx &c, size_t col,
-                                               const uint32_t (&g)[32], const uint32_t (&u)[32]) {
-  uint4 out[4];
+// Stage 1: SiLU(gate) * up for 32 columns held in registers, packed to bf16 (16 words).
+__device__ __forceinline__ void swiglu_pack32(const uint32_t (&g)[32], const uint32_t (&u)[32], uint4 (&out)[4]) {
   uint32_t *o = reinterpret_cast<uint32_t *>(out);
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
@@ -267,28 +269,38 @@ __device__ __forceinline__ void store_swiglu32(const TcParams &p, const Seg &S, 
                                               silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1])));
     o[i] = *reinterpret_cast<uint32_t *>(&h2);
   }
-  if (S.row_token && c.dst_in_regs) {
-#pragma unroll
-    for (int j = 0; j < kDstRegs; ++j) {
-      if (j < c.nd) {
-        uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)c.dst[j] * S.ldu + col);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) d4[q] = out[q];
-      }
-    }
-  } else if (S.row_token) {
-    // more paths per token than destination registers: look the copies up again
-    for (int k = 0; k < p.K; ++k) {
-      if (S.path_prow1[(size_t)c.token * p.K + k] != c.my_prow) continue;
-      uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)S.path_pos2[(size_t)c.token * p.K + k] * S.ldu + col);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) d4[q] = out[q];
-    }
-  } else {
-    uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)c.my_prow * S.ldu + col);
+}
+
+// Direct store of 32 bf16 of this thread's row to every path that reuses it, looked up on the spot
+// (only when a token has more paths than the destination registers hold).
+__device__ __forceinline__ void store_row_lookup(const TcParams &p, const Seg &S, const RowCtx &c, size_t col,
+                                                 const uint4 (&out)[4]) {
+  for (int k = 0; k < p.K; ++k) {
+    if (S.path_prow1[(size_t)c.token * p.K + k] != c.my_prow) continue;
+    uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)S.path_pos2[(size_t)c.token * p.K + k] * S.ldu + col);
 #pragma unroll
     for (int q = 0; q < 4; ++q) d4[q] = out[q];
   }
+}
+
+
+// Stage 2: this lane's 32 values (one row) are scaled by the path weight, staged, and added to y row by row.
+__device__ __forceinline__ void scatter_add_32x32(const TcParams &p, float *stage, const uint32_t (&v)[32], float wgt,
+                                                  int tok_or_neg, float *ycol, int lane) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    *reinterpret_cast<float4 *>(stage + lane * kEpiStride + 4 * q) =
+        make_float4(wgt * __uint_as_float(v[4 * q]), wgt * __uint_as_float(v[4 * q + 1]),
+                    wgt * __uint_as_float(v[4 * q + 2]), wgt * __uint_as_float(v[4 * q + 3]));
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = i * 4 + (lane >> 3);
+    const int tok = __shfl_sync(0xffffffffu, tok_or_neg, row);
+    const float4 x = *reinterpret_cast<const float4 *>(stage + row * kEpiStride + 4 * (lane & 7));
+    if (tok >= 0) red_add_v4(ycol + (size_t)tok * p.ldy, x.x, x.y, x.z, x.w);
+  }
+  __syncwarp();
 }
 
 // Drains one accumulator (this thread's TMEM lane) and applies the stage's epilogue.  TMEM loads are issued
@@ -296,29 +308,61 @@ __device__ __forceinline__ void store_swiglu32(const TcParams &p, const Seg &S, 
 // long while the next tile is being computed, and must overlap the math and the stores of the previous step.
 template <int STAGE>
 __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, const TileInfo &t, const RowCtx &c,
-                                              uint32_t taddr) {
+                                              uint32_t taddr, float *stage) {
   if (STAGE == 1) {
+    // 32 rows x 64 bf16 columns are collected in shared memory, then every destination row receives its
+    // 128 contiguous bytes from eight lanes (whole lines), four rows per instruction.
+    const int lane = threadIdx.x & 31;
     const size_t col0 = (size_t)t.n_idx * 128;
+    const int max_nd = c.dst_in_regs ? __reduce_max_sync(0xffffffffu, c.nd) : 0;
+    unsigned char *srow = reinterpret_cast<unsigned char *>(stage) + lane * (kEpiStride * 4);
     uint32_t g0[32], u0[32], g1[32], u1[32];
     tmem_ld32_issue(taddr, g0);
     tmem_ld32_issue(taddr + 128, u0);
 #pragma unroll
     for (int c0 = 0; c0 < 128; c0 += 64) {
+      uint4 out[4];
       tmem_wait_ld();
       reg_fence32(g0); reg_fence32(u0);
       tmem_ld32_issue(taddr + c0 + 32, g1);
       tmem_ld32_issue(taddr + 128 + c0 + 32, u1);
-      if (c.ok) store_swiglu32(p, S, c, col0 + c0, g0, u0);
+      swiglu_pack32(g0, u0, out);
+      if (c.ok && !c.dst_in_regs) store_row_lookup(p, S, c, col0 + c0, out);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow)[q] = out[q];
       tmem_wait_ld();
       reg_fence32(g1); reg_fence32(u1);
       if (c0 + 64 < 128) {
         tmem_ld32_issue(taddr + c0 + 64, g0);
         tmem_ld32_issue(taddr + 128 + c0 + 64, u0);
       }
-      if (c.ok) store_swiglu32(p, S, c, col0 + c0 + 32, g1, u1);
+      swiglu_pack32(g1, u1, out);
+      if (c.ok && !c.dst_in_regs) store_row_lookup(p, S, c, col0 + c0 + 32, out);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow + 64)[q] = out[q];
+      __syncwarp();
+      for (int k = 0; k < max_nd; ++k) {
+        int dk = -1;
+#pragma unroll
+        for (int j = 0; j < kDstRegs; ++j)
+          if (j == k && k < c.nd) dk = c.dst[j];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int row = i * 4 + (lane >> 3);
+          const int d = __shfl_sync(0xffffffffu, dk, row);
+          const uint4 x = *reinterpret_cast<const uint4 *>(reinterpret_cast<unsigned char *>(stage) +
+                                                           row * (kEpiStride * 4) + (lane & 7) * 16);
+          if (d >= 0) *reinterpret_cast<uint4 *>(S.u_out + (size_t)d * S.ldu + col0 + c0 + (lane & 7) * 8) = x;
+        }
+      }
+      __syncwarp();
     }
   } else {
-    float *dst = p.y + (size_t)c.token * p.ldy + (size_t)t.n_idx * 256;
+    // The warp's 32 rows x 32 columns are turned around in shared memory so that one instruction adds
+    // 128 contiguous bytes to each of four token rows (whole lines) instead of 16 bytes to 32 rows.
+    const int lane = threadIdx.x & 31;
+    const int tok_or_neg = c.ok ? c.token : -1;
+    float *ybase = p.y + (size_t)t.n_idx * 256 + 4 * (lane & 7);
     uint32_t v0[32], v1[32];
     tmem_ld32_issue(taddr, v0);
 #pragma unroll 1
@@ -326,21 +370,11 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
       tmem_wait_ld();
       reg_fence32(v0);
       tmem_ld32_issue(taddr + c0 + 32, v1);
-      if (c.ok) {
-#pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          red_add_v4(dst + c0 + i, c.wgt * __uint_as_float(v0[i]), c.wgt * __uint_as_float(v0[i + 1]),
-                     c.wgt * __uint_as_float(v0[i + 2]), c.wgt * __uint_as_float(v0[i + 3]));
-      }
+      scatter_add_32x32(p, stage, v0, c.wgt, tok_or_neg, ybase + c0, lane);
       tmem_wait_ld();
       reg_fence32(v1);
       if (c0 + 64 < 256) tmem_ld32_issue(taddr + c0 + 64, v0);
-      if (c.ok) {
-#pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          red_add_v4(dst + c0 + 32 + i, c.wgt * __uint_as_float(v1[i]), c.wgt * __uint_as_float(v1[i + 1]),
-                     c.wgt * __uint_as_float(v1[i + 2]), c.wgt * __uint_as_float(v1[i + 3]));
-      }
+      scatter_add_32x32(p, stage, v1, c.wgt, tok_or_neg, ybase + c0 + 32, lane);
     }
   }
 }
@@ -358,6 +392,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
   __shared__ __align__(8) uint64_t s_bar[2 * STAGES + 4];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
+  __shared__ __align__(16) float s_epi[4 * 32 * kEpiStride];   // per epilogue warp: 32 rows being turned around
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;   // 1024-byte aligned for the swizzle
@@ -489,7 +524,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
       const RowCtx c = prepare_row<STAGE>(p, S, t, r);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16));
+      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
+                           s_epi + (warp - 2) * 32 * kEpiStride);
       tc_fence_before();
       mbar_arrive(acce_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -617,6 +653,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   __shared__ __align__(8) uint64_t s_bar[2 * STAGES2 + 4];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
+  __shared__ __align__(16) float s_epi[4 * 32 * kEpiStride];   // per epilogue warp: 32 rows being turned around
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
@@ -764,7 +801,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
       const RowCtx c = prepare_row<STAGE>(p, S, t, r);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16));
+      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
+                           s_epi + (warp - 2) * 32 * kEpiStride);
       tc_fence_before();
       mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));   // the leader's MMA waits for both halves
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
