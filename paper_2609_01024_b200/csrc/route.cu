@@ -4,7 +4,8 @@
 //     s_a = (z[i] + b_ij) + lambda * u[j],
 // with three separately rounded fp32 operations, keeps the K best under the total order
 // (score descending, flat id ascending) - the TopK of Sec. 4.3 over the active set only -
-// and turns the selected scores into path weights with a softmax.
+// and turns the selected scores into path weights with a softmax.  The selection first filters the
+// paths with a warp-wide threshold and ranks the few survivors; heavy ties use per-lane sorted lists.
 #include <cfloat>
 
 #include "common.cuh"
@@ -22,6 +23,7 @@ struct RouteParams {
   float lambda, scale;
   int32_t norm_topk;
   int32_t table_in_smem;
+  int32_t cache_scores;      // pass 1 keeps the scores in shared memory for pass 2
 };
 
 __device__ __forceinline__ float path_score(const ActiveEntry e, const float *zs, const float *us,
@@ -36,21 +38,94 @@ __device__ __forceinline__ bool ranks_before(float s1, int a1, float s2, int a2)
   return s1 > s2 || (s1 == s2 && a1 < a2);
 }
 
+// Exact TopK by per-lane sorted lists: every lane keeps the best KMAX of its own entries (ties keep the
+// smaller table index first, because a lane visits its entries in ascending order and only a strictly
+// larger score moves up), then K rounds of a warp arg-max over the list heads pop the winners.
+// Lane k returns the k-th selection.  Used when the threshold filter below finds too many candidates.
+template <int KMAX>
+__device__ __noinline__ void topk_by_lists(const RouteParams &p, const ActiveEntry *tab, const float *zs,
+                                           const float *us, int lane, float &my_s, int &my_a) {
+  float ls[KMAX];
+  int la[KMAX];
+#pragma unroll
+  for (int i = 0; i < KMAX; ++i) {
+    ls[i] = -FLT_MAX;
+    la[i] = 0x7fffffff;
+  }
+  for (int a = lane; a < p.A; a += 32) {
+    const float s = path_score(tab[a], zs, us, p.lambda);
+    if (s > ls[KMAX - 1] || la[KMAX - 1] == 0x7fffffff) {
+      ls[KMAX - 1] = s;
+      la[KMAX - 1] = a;
+#pragma unroll
+      for (int i = KMAX - 1; i > 0; --i) {
+        if (ranks_before(ls[i], la[i], ls[i - 1], la[i - 1])) {
+          float ts = ls[i]; ls[i] = ls[i - 1]; ls[i - 1] = ts;
+          int ta = la[i]; la[i] = la[i - 1]; la[i - 1] = ta;
+        }
+      }
+    }
+  }
+  for (int k = 0; k < p.K; ++k) {
+    float bs = ls[0];
+    int ba = la[0];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float os = __shfl_xor_sync(0xffffffffu, bs, off);
+      const int oa = __shfl_xor_sync(0xffffffffu, ba, off);
+      if (ranks_before(os, oa, bs, ba)) {
+        bs = os;
+        ba = oa;
+      }
+    }
+    if (la[0] == ba) {  // this lane owns the winner: pop it
+#pragma unroll
+      for (int i = 0; i < KMAX - 1; ++i) {
+        ls[i] = ls[i + 1];
+        la[i] = la[i + 1];
+      }
+      ls[KMAX - 1] = -FLT_MAX;
+      la[KMAX - 1] = 0x7fffffff;
+    }
+    if (lane == k) {
+      my_s = bs;
+      my_a = ba;
+    }
+  }
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+  return v;
+}
+
 template <int KMAX>
 __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int warps = blockDim.x >> 5;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float *zrows = reinterpret_cast<float *>(smem_raw);                 // [warps][2][n]
+  float *cand_all = zrows + (size_t)warps * 2 * p.n;                  // [warps][64]: 32 scores, 32 indices
   const ActiveEntry *tab = p.table;
   if (p.table_in_smem) {
-    ActiveEntry *st = reinterpret_cast<ActiveEntry *>(smem_raw + (((size_t)warps * 2 * p.n * 4 + 15) & ~size_t(15)));
+    ActiveEntry *st = reinterpret_cast<ActiveEntry *>(smem_raw + (((size_t)warps * (2 * p.n + 64) * 4 + 15) & ~size_t(15)));
     for (int a = threadIdx.x; a < p.A; a += blockDim.x) st[a] = p.table[a];
     tab = st;
     __syncthreads();
   }
   float *zs = zrows + (size_t)warp * 2 * p.n;
   float *us = zs + p.n;
+  float *cand_s = cand_all + warp * 64;
+  int *cand_a = reinterpret_cast<int *>(cand_s + 32);
+  const int rounds = (p.A + 31) >> 5;
+  // optional per-warp score cache behind the table: [warps][rounds*32]
+  float *cache = nullptr;
+  if (p.cache_scores) {
+    size_t off = ((size_t)warps * (2 * p.n + 64) * 4 + 15) & ~size_t(15);
+    if (p.table_in_smem) off += (sizeof(ActiveEntry) * (size_t)p.A + 15) & ~size_t(15);
+    cache = reinterpret_cast<float *>(smem_raw + off) + (size_t)warp * rounds * 32;
+  }
 
   for (int t = blockIdx.x * warps + warp; t < p.T; t += gridDim.x * warps) {
     __syncwarp();
@@ -60,58 +135,71 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
     }
     __syncwarp();
 
-    // per-lane sorted list of its best KMAX candidates (ties keep the smaller table index first,
-    // because a lane visits its entries in ascending order and only a strictly larger score moves up)
-    float ls[KMAX];
-    int la[KMAX];
-#pragma unroll
-    for (int i = 0; i < KMAX; ++i) {
-      ls[i] = -FLT_MAX;
-      la[i] = 0x7fffffff;
-    }
+    // Threshold filter.  tau = the K-th largest of the 32 per-lane maxima: at least K paths score >= tau,
+    // so every path of the TopK scores >= tau, and usually only a handful of paths do.  Those candidates
+    // (ties with tau included) are compacted one per lane and ranked exactly; when more than 32 qualify
+    // (heavy ties) the token falls back to the per-lane lists, which give the same selection.
+    float m = -FLT_MAX;
     for (int a = lane; a < p.A; a += 32) {
       const float s = path_score(tab[a], zs, us, p.lambda);
-      if (s > ls[KMAX - 1] || la[KMAX - 1] == 0x7fffffff) {
-        ls[KMAX - 1] = s;
-        la[KMAX - 1] = a;
-#pragma unroll
-        for (int i = KMAX - 1; i > 0; --i) {
-          if (ranks_before(ls[i], la[i], ls[i - 1], la[i - 1])) {
-            float ts = ls[i]; ls[i] = ls[i - 1]; ls[i - 1] = ts;
-            int ta = la[i]; la[i] = la[i - 1]; la[i - 1] = ta;
-          }
+      if (cache) cache[a] = s;
+      m = fmaxf(m, s);
+    }
+    float tau = 0.0f;
+    for (int k = 0; k < p.K; ++k) {
+      tau = warp_max(m);
+      const unsigned hit = __ballot_sync(0xffffffffu, m == tau);
+      if (lane == __ffs(hit) - 1) m = -FLT_MAX;
+    }
+    int cnt = 0;
+    for (int i = 0; i < rounds; ++i) {
+      const int a = (i << 5) + lane;
+      float s = 0.0f;
+      bool q = false;
+      if (a < p.A) {
+        s = cache ? cache[a] : path_score(tab[a], zs, us, p.lambda);
+        q = s >= tau;
+      }
+      const unsigned b = __ballot_sync(0xffffffffu, q);
+      if (q) {
+        const int pos = cnt + __popc(b & ((1u << lane) - 1u));
+        if (pos < 32) {
+          cand_s[pos] = s;
+          cand_a[pos] = a;
         }
       }
+      cnt += __popc(b);
     }
+    __syncwarp();
 
-    // K rounds of warp arg-max over the lane heads
     float my_s = -FLT_MAX;
     int my_a = 0;
-    for (int k = 0; k < p.K; ++k) {
-      float bs = ls[0];
-      int ba = la[0];
+    if (cnt <= 32) {
+      float cs = lane < cnt ? cand_s[lane] : -FLT_MAX;
+      int ca = lane < cnt ? cand_a[lane] : 0x7fffffff;
+      for (int k = 0; k < p.K; ++k) {
+        float bs = cs;
+        int ba = ca;
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        const float os = __shfl_xor_sync(0xffffffffu, bs, off);
-        const int oa = __shfl_xor_sync(0xffffffffu, ba, off);
-        if (ranks_before(os, oa, bs, ba)) {
-          bs = os;
-          ba = oa;
+        for (int off = 16; off > 0; off >>= 1) {
+          const float os = __shfl_xor_sync(0xffffffffu, bs, off);
+          const int oa = __shfl_xor_sync(0xffffffffu, ba, off);
+          if (ranks_before(os, oa, bs, ba)) {
+            bs = os;
+            ba = oa;
+          }
+        }
+        if (ca == ba) {
+          cs = -FLT_MAX;
+          ca = 0x7fffffff;
+        }
+        if (lane == k) {
+          my_s = bs;
+          my_a = ba;
         }
       }
-      if (la[0] == ba) {  // this lane owns the winner: pop it
-#pragma unroll
-        for (int i = 0; i < KMAX - 1; ++i) {
-          ls[i] = ls[i + 1];
-          la[i] = la[i + 1];
-        }
-        ls[KMAX - 1] = -FLT_MAX;
-        la[KMAX - 1] = 0x7fffffff;
-      }
-      if (lane == k) {
-        my_s = bs;
-        my_a = ba;
-      }
+    } else {
+      topk_by_lists<KMAX>(p, tab, zs, us, lane, my_s, my_a);
     }
 
     const float s0 = __shfl_sync(0xffffffffu, my_s, 0);
@@ -144,10 +232,13 @@ pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, con
   p.T = T; p.n = c.n_experts; p.K = c.top_k; p.A = L->n_active;
   p.lambda = c.lambda; p.scale = c.routed_scale; p.norm_topk = c.norm_topk;
   const int threads = 256, warps = threads / 32;
-  size_t smem = ((size_t)warps * 2 * p.n * 4 + 15) & ~size_t(15);
+  size_t smem = ((size_t)warps * (2 * p.n + 64) * 4 + 15) & ~size_t(15);
   const size_t tab_bytes = sizeof(ActiveEntry) * (size_t)p.A;
   p.table_in_smem = smem + tab_bytes <= 160 * 1024;
-  if (p.table_in_smem) smem += tab_bytes;
+  if (p.table_in_smem) smem += (tab_bytes + 15) & ~size_t(15);
+  const size_t cache_bytes = (size_t)warps * ((p.A + 31) / 32 * 32) * 4;
+  p.cache_scores = smem + cache_bytes <= 100 * 1024;
+  if (p.cache_scores) smem += cache_bytes;
   int grid = (T + warps - 1) / warps;
   const int cap = L->sm_count * 4;
   if (grid > cap) grid = cap;
