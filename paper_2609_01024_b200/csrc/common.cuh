@@ -71,6 +71,14 @@ void count_launch(int n = 1);
 
 inline size_t dtype_size(int dt) { return dt == PCOMOE_BF16 ? 2 : 4; }
 
+// Tokens per block of the grouping kernels for a batch of T tokens: the largest chunk the layer allows
+// (shared-memory bound), halved while that would leave fewer than two blocks per SM.
+inline int group_chunk_for(const pcomoe_layer *L, int32_t T) {
+  int chunk = L->group_chunk;
+  while (chunk > 32 && (int64_t)T / chunk < 2 * (int64_t)L->sm_count) chunk >>= 1;
+  return chunk;
+}
+
 #define PCOMOE_CUDA_TRY(expr)                          \
   do {                                                 \
     cudaError_t _e = (expr);                           \

@@ -825,15 +825,28 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   }
 }
 
-// Copies rows idx[r] of src into consecutive rows of dst (the gather-free fallback of the A operand).
-__global__ void gather_rows_kernel(uint4 *dst, const uint4 *src, const int32_t *idx, const int32_t *tile_base,
-                                   int G, int vec_per_row) {
+// Copies rows idx[r] of src into consecutive rows of dst (the A operand of stage 1 in group order).
+// One warp per row; a lane keeps up to eight 16-byte loads in flight before it stores.
+__global__ void __launch_bounds__(256) gather_rows_kernel(uint4 *dst, const uint4 *src, const int32_t *idx,
+                                                          const int32_t *tile_base, int G, int vec_per_row) {
   const int rows = tile_base[G] * kTileM;
-  const int warps_per_block = blockDim.x >> 5;
+  const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
   for (int r = blockIdx.x * warps_per_block + (threadIdx.x >> 5); r < rows; r += gridDim.x * warps_per_block) {
     const uint4 *s = src + (size_t)idx[r] * vec_per_row;
     uint4 *d = dst + (size_t)r * vec_per_row;
-    for (int v = threadIdx.x & 31; v < vec_per_row; v += 32) d[v] = s[v];
+    for (int v0 = 0; v0 < vec_per_row; v0 += 256) {
+      uint4 x[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int v = v0 + i * 32 + lane;
+        if (v < vec_per_row) x[i] = __ldg(s + v);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int v = v0 + i * 32 + lane;
+        if (v < vec_per_row) d[v] = x[i];
+      }
+    }
   }
 }
 
@@ -914,7 +927,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     int ns = 0;
     bool ok = true;
     if (stages & kStage1Routed) {
-      gather_rows_kernel<<<L->sm_count * 4, 256, 0, st>>>(Hg, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
+      gather_rows_kernel<<<L->sm_count * 8, 256, 0, st>>>(Hg, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
       count_launch();
       ok = ok && make_map(&mA[ns], Hg, pad_rows, H, kTileM) && make_map(&mB[ns], wg, (uint64_t)n * F, H, 128) &&
            make_map(&mC[ns], wu, (uint64_t)n * F, H, 128);

@@ -20,7 +20,7 @@ struct GroupParams {
   pcomoe_groups g;
   DevPlan *plan;
   int32_t *tile_base1, *tile_base2;   // [n+1]
-  int32_t *blk_cnt;                   // [NB][2][n]
+  int32_t *blk_cnt;                   // [2][n][NB]: per-block counts, turned into per-block offsets by the scan
   int32_t *a1_idx;                    // token of every padded stage-1 row
   int32_t *path_prow1, *path_pos2;    // [T,K] padded stage-1 / stage-2 row of every path
   int32_t T, n, K, dedup, chunk, nb;
@@ -69,8 +69,7 @@ __global__ void group_count_kernel(const GroupParams p) {
     }
   }
   __syncthreads();
-  int32_t *out = p.blk_cnt + (size_t)blockIdx.x * 2 * p.n;
-  for (int e = threadIdx.x; e < 2 * p.n; e += blockDim.x) out[e] = h1[e];
+  for (int e = threadIdx.x; e < 2 * p.n; e += blockDim.x) p.blk_cnt[(size_t)e * p.nb + blockIdx.x] = h1[e];
 }
 
 __device__ __forceinline__ int warp_incl_scan(int v, int lane) {
@@ -85,14 +84,30 @@ __device__ __forceinline__ int warp_incl_scan(int v, int lane) {
 __global__ void __launch_bounds__(1024) group_scan_kernel(const GroupParams p) {
   __shared__ int32_t tot[2 * kMaxExperts];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
-  // (stage, expert) columns: exclusive prefix over the blocks, in place
+  // (stage, expert) columns: exclusive prefix over the blocks, in place.  A lane owns a contiguous run of
+  // blocks, so all its loads are issued at once; the warp then scans the lane totals.
+  constexpr int kRun = 8;
   for (int col = warp; col < 2 * p.n; col += warps) {
+    int32_t *c = p.blk_cnt + (size_t)col * p.nb;
     int carry = 0;
-    for (int b0 = 0; b0 < p.nb; b0 += 32) {
-      const int b = b0 + lane;
-      const int v = b < p.nb ? p.blk_cnt[(size_t)b * 2 * p.n + col] : 0;
-      const int incl = warp_incl_scan(v, lane);
-      if (b < p.nb) p.blk_cnt[(size_t)b * 2 * p.n + col] = carry + incl - v;
+    for (int b0 = 0; b0 < p.nb; b0 += 32 * kRun) {
+      int v[kRun];
+#pragma unroll
+      for (int i = 0; i < kRun; ++i) {
+        const int b = b0 + lane * kRun + i;
+        v[i] = b < p.nb ? c[b] : 0;
+      }
+      int sum = 0;
+#pragma unroll
+      for (int i = 0; i < kRun; ++i) sum += v[i];
+      const int incl = warp_incl_scan(sum, lane);
+      int run = carry + incl - sum;
+#pragma unroll
+      for (int i = 0; i < kRun; ++i) {
+        const int b = b0 + lane * kRun + i;
+        if (b < p.nb) c[b] = run;
+        run += v[i];
+      }
       carry += __shfl_sync(0xffffffffu, incl, 31);
     }
     if (lane == 0) tot[col] = carry;
@@ -152,14 +167,13 @@ __global__ void group_scatter_kernel(const GroupParams p) {
   uint32_t *bits1 = reinterpret_cast<uint32_t *>(bo2 + p.n), *bits2 = bits1 + (size_t)p.n * W;
 
   for (int x = threadIdx.x; x < 2 * p.n * W; x += blockDim.x) bits1[x] = 0u;
-  const int32_t *bo = p.blk_cnt + (size_t)blockIdx.x * 2 * p.n;
   for (int e = threadIdx.x; e < p.n; e += blockDim.x) {
     off1[e] = p.g.s1_offsets[e];
     off2[e] = p.g.s2_offsets[e];
     tb1[e] = p.tile_base1[e];
     tb2[e] = p.tile_base2[e];
-    bo1[e] = bo[e];
-    bo2[e] = bo[p.n + e];
+    bo1[e] = p.blk_cnt[(size_t)e * p.nb + blockIdx.x];
+    bo2[e] = p.blk_cnt[(size_t)(p.n + e) * p.nb + blockIdx.x];
   }
   const int nt = stage_chunk(p, ssrc, stgt);
   __syncthreads();
@@ -227,7 +241,7 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
   p.a1_idx = reinterpret_cast<int32_t *>(ws + lay.a1_idx);
   p.path_prow1 = reinterpret_cast<int32_t *>(ws + lay.path_prow1);
   p.path_pos2 = reinterpret_cast<int32_t *>(ws + lay.path_pos2);
-  p.T = T; p.n = c.n_experts; p.K = c.top_k; p.dedup = c.dedup; p.chunk = L->group_chunk;
+  p.T = T; p.n = c.n_experts; p.K = c.top_k; p.dedup = c.dedup; p.chunk = group_chunk_for(L, T);
   p.nb = (T + p.chunk - 1) / p.chunk;
 
   // the status word and the plan start from zero (the scan kernel fills the padding of the gather map)

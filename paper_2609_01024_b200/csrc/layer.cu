@@ -20,7 +20,10 @@ WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
   WsLayout w{};
   const int64_t Tm = max_tokens > 0 ? max_tokens : 1;
   const int64_t Pm = Tm * c.top_k;
-  w.nb_max = (int32_t)((Tm + L->group_chunk - 1) / L->group_chunk);
+  // upper bound of the grouping kernels' block count for any batch up to Tm (see group_chunk_for)
+  const int64_t nb_small = (Tm + 31) / 32 < 4 * (int64_t)L->sm_count ? (Tm + 31) / 32 : 4 * (int64_t)L->sm_count;
+  const int64_t nb_large = (Tm + L->group_chunk - 1) / L->group_chunk;
+  w.nb_max = (int32_t)(nb_small > nb_large ? nb_small : nb_large);
   w.mt_max = (int32_t)(Pm / kTileM + c.n_experts + 1);
   w.t_pad = (int32_t)((Tm + kTileM - 1) / kTileM * kTileM);
   const size_t es = dtype_size(c.in_dtype);
