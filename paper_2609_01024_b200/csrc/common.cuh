@@ -37,7 +37,8 @@ struct WsLayout {
   size_t plan;         // DevPlan
   size_t tile_base1;   // int32 [n+1]   prefix of stage-1 m-tiles per source
   size_t tile_base2;   // int32 [n+1]   prefix of stage-2 m-tiles per target
-  size_t blk_cnt;      // int32 [NB][2][n] per-block histograms, turned into offsets by the scan
+  size_t col_tot;      // int32 [2][n]     rows per (stage, expert)
+  size_t blk_cnt;      // int32 [2][n][NB] per-block histograms, turned into offsets by the scan
   size_t a1_idx;       // int32 [mt_max*128] token of every padded stage-1 row (0 in the padding)
   size_t path_prow1;   // int32 [T*K] padded stage-1 row of every path
   size_t path_pos2;    // int32 [T*K] padded stage-2 row of every path

@@ -3,9 +3,9 @@
 // A stable counting sort in three launches, bit-exact and free of inter-block waiting:
 //   count    each block histograms the sources (first occurrences only when reuse is on) and the
 //            targets of its contiguous chunk of tokens;
-//   scan     one block turns the per-block histograms into per-block offsets, the per-expert
-//            offsets, and the 128-row tile schedule of the two GEMM stages;
-//   scatter  each block ranks its own paths with a bit matrix [expert][flat id in chunk]
+//   colscan  one warp per (stage, expert) turns the per-block counts into per-block offsets and a total;
+//   scatter  each block derives the per-expert offsets and the 128-row tile schedule of the two GEMM stages
+//            from the totals (block 0 publishes them), ranks its own paths with a bit matrix [expert][flat id in chunk]
 //            (rank = set bits below mine) and writes every output at its final position.
 // Orders are canonical: stage-1 rows by (source, token) - or (source, flat path id) without
 // reuse - and stage-2 rows by (target, flat path id).
@@ -20,6 +20,7 @@ struct GroupParams {
   pcomoe_groups g;
   DevPlan *plan;
   int32_t *tile_base1, *tile_base2;   // [n+1]
+  int32_t *col_tot;                   // [2][n] rows per (stage, expert)
   int32_t *blk_cnt;                   // [2][n][NB]: per-block counts, turned into per-block offsets by the scan
   int32_t *a1_idx;                    // token of every padded stage-1 row
   int32_t *path_prow1, *path_pos2;    // [T,K] padded stage-1 / stage-2 row of every path
@@ -81,71 +82,78 @@ __device__ __forceinline__ int warp_incl_scan(int v, int lane) {
   return v;
 }
 
-__global__ void __launch_bounds__(1024) group_scan_kernel(const GroupParams p) {
-  __shared__ int32_t tot[2 * kMaxExperts];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
-  // (stage, expert) columns: exclusive prefix over the blocks, in place.  A lane owns a contiguous run of
-  // blocks, so all its loads are issued at once; the warp then scans the lane totals.
+// One warp per (stage, expert) column: exclusive prefix of the per-block counts over the blocks, in place,
+// and the column total.  A lane owns a contiguous run of blocks, so all its loads are issued at once.
+__global__ void __launch_bounds__(128) group_colscan_kernel(const GroupParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int col = blockIdx.x * (blockDim.x >> 5) + warp;
+  if (col >= 2 * p.n) return;
   constexpr int kRun = 8;
-  for (int col = warp; col < 2 * p.n; col += warps) {
-    int32_t *c = p.blk_cnt + (size_t)col * p.nb;
-    int carry = 0;
-    for (int b0 = 0; b0 < p.nb; b0 += 32 * kRun) {
-      int v[kRun];
+  int32_t *c = p.blk_cnt + (size_t)col * p.nb;
+  int carry = 0;
+  for (int b0 = 0; b0 < p.nb; b0 += 32 * kRun) {
+    int v[kRun];
 #pragma unroll
-      for (int i = 0; i < kRun; ++i) {
-        const int b = b0 + lane * kRun + i;
-        v[i] = b < p.nb ? c[b] : 0;
-      }
-      int sum = 0;
-#pragma unroll
-      for (int i = 0; i < kRun; ++i) sum += v[i];
-      const int incl = warp_incl_scan(sum, lane);
-      int run = carry + incl - sum;
-#pragma unroll
-      for (int i = 0; i < kRun; ++i) {
-        const int b = b0 + lane * kRun + i;
-        if (b < p.nb) c[b] = run;
-        run += v[i];
-      }
-      carry += __shfl_sync(0xffffffffu, incl, 31);
+    for (int i = 0; i < kRun; ++i) {
+      const int b = b0 + lane * kRun + i;
+      v[i] = b < p.nb ? c[b] : 0;
     }
-    if (lane == 0) tot[col] = carry;
+    int sum = 0;
+#pragma unroll
+    for (int i = 0; i < kRun; ++i) sum += v[i];
+    const int incl = warp_incl_scan(sum, lane);
+    int run = carry + incl - sum;
+#pragma unroll
+    for (int i = 0; i < kRun; ++i) {
+      const int b = b0 + lane * kRun + i;
+      if (b < p.nb) c[b] = run;
+      run += v[i];
+    }
+    carry += __shfl_sync(0xffffffffu, incl, 31);
   }
-  __syncthreads();
-  // warp 0: stage 1, warp 1: stage 2.  Offsets over the experts and the m-tile schedule.
-  if (warp < 2) {
-    const int32_t *cnt = tot + warp * p.n;
-    int32_t *offs = warp == 0 ? p.g.s1_offsets : p.g.s2_offsets;
-    int32_t *tb = warp == 0 ? p.tile_base1 : p.tile_base2;
-    int carry_rows = 0, carry_tiles = 0, empty = 0;
-    for (int e0 = 0; e0 < p.n; e0 += 32) {
-      const int e = e0 + lane;
-      const int c = e < p.n ? cnt[e] : 0;
-      const int tl = (c + kTileM - 1) / kTileM;
-      const int ir = warp_incl_scan(c, lane), it = warp_incl_scan(tl, lane);
-      if (e < p.n) {
-        offs[e] = carry_rows + ir - c;
-        tb[e] = carry_tiles + it - tl;
-        if (warp == 0)  // the padding rows of a source group gather token 0 (any valid row will do)
-          for (int x = c; x < tl * kTileM; ++x) p.a1_idx[(size_t)(carry_tiles + it - tl) * kTileM + x] = 0;
+  if (lane == 0) p.col_tot[col] = carry;
+}
+
+// Offsets over the experts and the 128-row tile schedule of one stage, from the column totals (one warp).
+// Every scatter block computes them for itself; block 0 also publishes them, the statistics, and the
+// padding entries of the stage-1 gather map.
+__device__ __forceinline__ void expert_prefix(const GroupParams &p, int stage, int32_t *offs_s, int32_t *tb_s,
+                                              bool publish, int lane) {
+  const int32_t *cnt = p.col_tot + stage * p.n;
+  int32_t *offs = stage == 0 ? p.g.s1_offsets : p.g.s2_offsets;
+  int32_t *tb = stage == 0 ? p.tile_base1 : p.tile_base2;
+  int carry_rows = 0, carry_tiles = 0, empty = 0;
+  for (int e0 = 0; e0 < p.n; e0 += 32) {
+    const int e = e0 + lane;
+    const int c = e < p.n ? cnt[e] : 0;
+    const int tl = (c + kTileM - 1) / kTileM;
+    const int ir = warp_incl_scan(c, lane), it = warp_incl_scan(tl, lane);
+    if (e < p.n) {
+      const int o = carry_rows + ir - c, t0 = carry_tiles + it - tl;
+      offs_s[e] = o;
+      tb_s[e] = t0;
+      if (publish) {
+        offs[e] = o;
+        tb[e] = t0;
+        if (stage == 0)  // the padding rows of a source group gather token 0 (any valid row will do)
+          for (int x = c; x < tl * kTileM; ++x) p.a1_idx[(size_t)t0 * kTileM + x] = 0;
       }
-      empty += __popc(__ballot_sync(0xffffffffu, e < p.n && c == 0));
-      carry_rows += __shfl_sync(0xffffffffu, ir, 31);
-      carry_tiles += __shfl_sync(0xffffffffu, it, 31);
     }
-    if (lane == 0) {
-      offs[p.n] = carry_rows;
-      tb[p.n] = carry_tiles;
-      if (warp == 0) {
-        p.plan->R1 = carry_rows; p.plan->mt1 = carry_tiles; p.plan->empty1 = empty;
-        p.plan->T = p.T;
-        p.g.stats[0] = carry_rows; p.g.stats[2] = carry_tiles; p.g.stats[4] = empty;
-        p.g.stats[6] = 0; p.g.stats[7] = 0;
-      } else {
-        p.plan->P = carry_rows; p.plan->mt2 = carry_tiles; p.plan->empty2 = empty;
-        p.g.stats[1] = carry_rows; p.g.stats[3] = carry_tiles; p.g.stats[5] = empty;
-      }
+    empty += __popc(__ballot_sync(0xffffffffu, e < p.n && c == 0));
+    carry_rows += __shfl_sync(0xffffffffu, ir, 31);
+    carry_tiles += __shfl_sync(0xffffffffu, it, 31);
+  }
+  if (publish && lane == 0) {
+    offs[p.n] = carry_rows;
+    tb[p.n] = carry_tiles;
+    if (stage == 0) {
+      p.plan->R1 = carry_rows; p.plan->mt1 = carry_tiles; p.plan->empty1 = empty;
+      p.plan->T = p.T;
+      p.g.stats[0] = carry_rows; p.g.stats[2] = carry_tiles; p.g.stats[4] = empty;
+      p.g.stats[6] = 0; p.g.stats[7] = 0;
+    } else {
+      p.plan->P = carry_rows; p.plan->mt2 = carry_tiles; p.plan->empty2 = empty;
+      p.g.stats[1] = carry_rows; p.g.stats[3] = carry_tiles; p.g.stats[5] = empty;
     }
   }
 }
@@ -167,15 +175,17 @@ __global__ void group_scatter_kernel(const GroupParams p) {
   uint32_t *bits1 = reinterpret_cast<uint32_t *>(bo2 + p.n), *bits2 = bits1 + (size_t)p.n * W;
 
   for (int x = threadIdx.x; x < 2 * p.n * W; x += blockDim.x) bits1[x] = 0u;
-  for (int e = threadIdx.x; e < p.n; e += blockDim.x) {
-    off1[e] = p.g.s1_offsets[e];
-    off2[e] = p.g.s2_offsets[e];
-    tb1[e] = p.tile_base1[e];
-    tb2[e] = p.tile_base2[e];
-    bo1[e] = p.blk_cnt[(size_t)e * p.nb + blockIdx.x];
-    bo2[e] = p.blk_cnt[(size_t)(p.n + e) * p.nb + blockIdx.x];
+  if (threadIdx.x < 32) {
+    expert_prefix(p, 0, off1, tb1, blockIdx.x == 0, threadIdx.x);
+    expert_prefix(p, 1, off2, tb2, blockIdx.x == 0, threadIdx.x);
   }
-  const int nt = stage_chunk(p, ssrc, stgt);
+  if (p.nb > 0) {
+    for (int e = threadIdx.x; e < p.n; e += blockDim.x) {
+      bo1[e] = p.blk_cnt[(size_t)e * p.nb + blockIdx.x];
+      bo2[e] = p.blk_cnt[(size_t)(p.n + e) * p.nb + blockIdx.x];
+    }
+  }
+  const int nt = p.nb > 0 ? stage_chunk(p, ssrc, stgt) : 0;
   __syncthreads();
 
   const int tl = threadIdx.x;
@@ -238,6 +248,7 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
   p.tile_base1 = reinterpret_cast<int32_t *>(ws + lay.tile_base1);
   p.tile_base2 = reinterpret_cast<int32_t *>(ws + lay.tile_base2);
   p.blk_cnt = reinterpret_cast<int32_t *>(ws + lay.blk_cnt);
+  p.col_tot = reinterpret_cast<int32_t *>(ws + lay.col_tot);
   p.a1_idx = reinterpret_cast<int32_t *>(ws + lay.a1_idx);
   p.path_prow1 = reinterpret_cast<int32_t *>(ws + lay.path_prow1);
   p.path_pos2 = reinterpret_cast<int32_t *>(ws + lay.path_pos2);
@@ -260,12 +271,9 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
     group_count_kernel<<<p.nb, p.chunk, smem_count, st>>>(p);
     count_launch();
   }
-  group_scan_kernel<<<1, 1024, 0, st>>>(p);
-  count_launch();
-  if (p.nb > 0) {
-    group_scatter_kernel<<<p.nb, p.chunk, smem_scatter, st>>>(p);
-    count_launch();
-  }
+  group_colscan_kernel<<<(2 * p.n + 3) / 4, 128, 0, st>>>(p);
+  group_scatter_kernel<<<p.nb > 0 ? p.nb : 1, p.chunk, smem_scatter, st>>>(p);
+  count_launch(2);
   PCOMOE_CUDA_TRY(cudaGetLastError());
   return PCOMOE_OK;
 }

@@ -36,6 +36,7 @@ WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
   w.plan = take(sizeof(DevPlan));
   w.tile_base1 = take(sizeof(int32_t) * (c.n_experts + 1));
   w.tile_base2 = take(sizeof(int32_t) * (c.n_experts + 1));
+  w.col_tot = take(sizeof(int32_t) * 2 * c.n_experts);
   w.blk_cnt = take(sizeof(int32_t) * (size_t)w.nb_max * 2 * c.n_experts);
   w.a1_idx = take(sizeof(int32_t) * (size_t)w.mt_max * kTileM);
   w.path_prow1 = take(sizeof(int32_t) * (size_t)Pm);
