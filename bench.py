@@ -326,9 +326,9 @@ def main():
                "stage_ms": stage_ms}
         if not args.no_cpu_baseline and world == 1:
             n_cpu = args.cpu_tokens
-            if n_cpu <= 0:   # probe with a few tokens, then size the sample for about 15 s
-                r0, _, s0, nt0 = oracle_sample_rate(cfg, L, 8)
-                n_cpu = int(max(8, min(cfg.T, 15.0 * r0)))
+            if n_cpu <= 0:   # probe with a few tokens per thread, then size the sample for about 20 s
+                r0, _, s0, nt0 = oracle_sample_rate(cfg, L, 32)
+                n_cpu = int(max(32, min(cfg.T, 20.0 * r0)))
             r, thr, secs, nt = oracle_sample_rate(cfg, L, n_cpu)
             out["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": thr, "kind": "oracle",
                                    "sample": f"routing+grouping on all {cfg.T} tokens, FFN on {nt} seeded tokens ({secs:.1f} s)"}
