@@ -30,6 +30,9 @@ from paper_2609_01024_b200 import workloads as wl  # noqa: E402
 
 METRIC = "path_moe_layer_tokens_per_s"
 UNIT = "tokens/s"
+# DRAM bytes (dram__bytes_read + dram__bytes_write) of ONE launch of the dominant kernel (stage-1 grouped GEMM) on
+# the benchmark layers, from the ncu capture summarised in profiles/kernels_per_config.md
+NCU_TRAFFIC_STAGE1 = {2: 2340.7e6, 3: 1212.1e6, 4: 2047.5e6, 5: 1902.3e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -294,7 +297,8 @@ def main():
         ach = work["flops_s1"] / (stage_ms["stage1_routed"] * 1e-3) / 1e12
         peak = pk["bf16_tflops_sustained"]
         roofline = {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                    "traffic": None, "kernel": "grouped_gemm_kernel<1> (stage 1, routed groups)",
+                    "traffic": NCU_TRAFFIC_STAGE1.get(args.config) if not args.shape and args.variant == "default" else None,
+                    "kernel": "stage-1 grouped GEMM over the routed groups (row gather + grouped_gemm_pair_kernel<1>)",
                     "peak_source": pk["source"] + " sustained bf16 (kernel timed inside a loop of steps)"}
     else:
         # decode-sized / tiny: weight streaming; report the two GEMM stages' bytes against HBM
@@ -302,7 +306,8 @@ def main():
         ach = s1_bytes / (stage_ms["stage1_routed"] * 1e-3) / 1e9
         peak = pk["hbm_gbs"]
         roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                    "traffic": None, "kernel": "stage 1, routed groups (weight streaming)",
+                    "traffic": NCU_TRAFFIC_STAGE1.get(args.config) if not args.shape and args.variant == "default" else None,
+                    "kernel": "stage-1 grouped GEMM, routed groups (weight streaming, grouped_gemm_kernel<1>)",
                     "peak_source": pk["source"] + " copy bandwidth"}
     # whole-layer roofline time: max(FLOPs / tensor peak, bytes / HBM peak)
     t_roof_meas = max(work["flops"] / (pk["bf16_tflops_sustained"] * 1e12), work["bytes"] / (pk["hbm_gbs"] * 1e9))
