@@ -26,6 +26,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2609_01024_b200 import replicas  # noqa: E402
 from paper_2609_01024_b200 import workloads as wl  # noqa: E402
 
 METRIC = "path_moe_layer_tokens_per_s"
@@ -198,12 +199,8 @@ def main():
 
     # Every rank holds a replica of the weights and its own batch of T tokens (token data parallel,
     # no collective on the data path); rank r draws its tokens with seed + 100*r.
-    cfg_r = cfg if rank == 0 else cfg.scaled(seed=cfg.seed)  # same weights on every rank
-    L = wl.make_layer(cfg_r)
-    if rank > 0:
-        cfg_tok = cfg.scaled(seed=cfg.seed + 100 * rank)
-        L.h = wl.make_hidden(cfg_tok)
-        L.logits = wl.make_logits(cfg_tok, wl.hidden_as_f32(cfg_tok, L.h) if cfg.logits == "router" else None)
+    L = wl.make_layer(cfg)                              # same mask, bias and weights on every rank
+    L.h, L.logits = replicas.rank_inputs(cfg, rank)     # its own batch of tokens
     mask = np.eye(cfg.n, dtype=np.uint8) if args.variant == "vanilla" else L.mask
     dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
     layer = B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=cfg.F, mask=mask, bias=L.bias,
@@ -249,12 +246,8 @@ def main():
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     assert layer.device_status() == 0, "device reported an error during the timed steps"
-    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_max = float(t_ms.item())
-    ms_per_step = ms_max / args.steps
-    value = world * cfg.T / (ms_per_step * 1e-3)
+    ms_per_step = replicas.max_over_ranks(ms, dev) / args.steps
+    value = replicas.whole_job_tokens_per_s(cfg.T, world, ms_per_step)
 
     # ---- end to end through host buffers (pinned H2D of inputs, D2H of y) ----
     for _ in range(2):
@@ -264,10 +257,7 @@ def main():
     for _ in range(args.steps):
         y_host = layer.forward_host(L.logits, L.h)
     torch.cuda.synchronize()
-    t_e2e = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
-    e2e_value = world * cfg.T * args.steps / float(t_e2e.item())
+    e2e_value = world * cfg.T * args.steps / replicas.max_over_ranks(time.perf_counter() - t0, dev)
     h2d = L.logits.nbytes + L.h.nbytes
     d2h = cfg.T * cfg.H * 4
 
