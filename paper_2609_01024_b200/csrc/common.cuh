@@ -76,6 +76,7 @@ inline size_t dtype_size(int dt) { return dt == PCOMOE_BF16 ? 2 : 4; }
 // (shared-memory bound), halved while that would leave fewer than two blocks per SM.
 inline int group_chunk_for(const pcomoe_layer *L, int32_t T) {
   int chunk = L->group_chunk;
+  if (T <= chunk) return chunk;   // the whole batch fits one block
   while (chunk > 32 && (int64_t)T / chunk < 2 * (int64_t)L->sm_count) chunk >>= 1;
   return chunk;
 }
@@ -85,6 +86,33 @@ inline int group_chunk_for(const pcomoe_layer *L, int32_t T) {
     cudaError_t _e = (expr);                           \
     if (_e != cudaSuccess) return PCOMOE_ERR_CUDA;     \
   } while (0)
+
+// Programmatic dependent launch.  Every kernel of the library begins with pdl_grid_wait(), which holds it until
+// the kernel before it in the stream has completed and its writes are visible, and then lets the kernel after it
+// start its own launch and prologue early (it will block in its own pdl_grid_wait()).  Launched with
+// launch_pdl(), consecutive kernels of a call overlap their launch latencies instead of adding them.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_grid_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 // launchers implemented in the kernel translation units
 pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, const float *u,

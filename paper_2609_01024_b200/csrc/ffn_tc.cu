@@ -388,6 +388,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
                     const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmC1,
                     const TcParams p) {
   extern __shared__ unsigned char smem_dyn[];
+  pdl_grid_wait();
   __shared__ int32_t s_tb[2 * (kMaxExperts + 2)], s_ro[2 * (kMaxExperts + 2)];
   __shared__ __align__(8) uint64_t s_bar[2 * STAGES + 4];
   __shared__ uint32_t s_tmem;
@@ -649,6 +650,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
                          const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmC1,
                          const TcParams p) {
   extern __shared__ unsigned char smem_dyn[];
+  pdl_grid_wait();
   __shared__ int32_t s_tb[2 * (kMaxExperts + 2)], s_ro[2 * (kMaxExperts + 2)], s_pb[2 * (kMaxExperts + 2)];
   __shared__ __align__(8) uint64_t s_bar[2 * STAGES2 + 4];
   __shared__ uint32_t s_tmem;
@@ -829,6 +831,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
 // One warp per row; a lane keeps up to eight 16-byte loads in flight before it stores.
 __global__ void __launch_bounds__(256) gather_rows_kernel(uint4 *dst, const uint4 *src, const int32_t *idx,
                                                           const int32_t *tile_base, int G, int vec_per_row) {
+  pdl_grid_wait();
   const int rows = tile_base[G] * kTileM;
   const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
   for (int r = blockIdx.x * warps_per_block + (threadIdx.x >> 5); r < rows; r += gridDim.x * warps_per_block) {
@@ -927,7 +930,8 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     int ns = 0;
     bool ok = true;
     if (stages & kStage1Routed) {
-      gather_rows_kernel<<<L->sm_count * 8, 256, 0, st>>>(Hg, reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8);
+      PCOMOE_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3(L->sm_count * 8), dim3(256), 0, st, Hg,
+                                 reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8));
       count_launch();
       ok = ok && make_map(&mA[ns], Hg, pad_rows, H, kTileM) && make_map(&mB[ns], wg, (uint64_t)n * F, H, 128) &&
            make_map(&mC[ns], wu, (uint64_t)n * F, H, 128);
@@ -948,10 +952,8 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
       p.zero_ptr = reinterpret_cast<float4 *>(y);
       p.zero_vec4 = (int64_t)T * H / 4;
     }
-    if (pair)
-      grouped_gemm_pair_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p);
-    else
-      grouped_gemm_kernel<1><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p);
+    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<1> : grouped_gemm_kernel<1>, dim3(grid), dim3(kThreads),
+                               kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
     count_launch();
   }
 
@@ -980,10 +982,8 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; }
     p.nseg = ns;
-    if (pair)
-      grouped_gemm_pair_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p);
-    else
-      grouped_gemm_kernel<2><<<grid, kThreads, kSmemDyn, st>>>(mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p);
+    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<2> : grouped_gemm_kernel<2>, dim3(grid), dim3(kThreads),
+                               kSmemDyn, st, mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p));
     count_launch();
   }
   PCOMOE_CUDA_TRY(cudaGetLastError());

@@ -56,6 +56,7 @@ __device__ __forceinline__ int first_occurrence(const int32_t *row, int k, int d
 
 __global__ void group_count_kernel(const GroupParams p) {
   extern __shared__ int32_t sm[];
+  pdl_grid_wait();
   int32_t *ssrc = sm, *stgt = sm + p.chunk * p.K;
   int32_t *h1 = stgt + p.chunk * p.K, *h2 = h1 + p.n;
   for (int e = threadIdx.x; e < 2 * p.n; e += blockDim.x) h1[e] = 0;
@@ -85,6 +86,7 @@ __device__ __forceinline__ int warp_incl_scan(int v, int lane) {
 // One warp per (stage, expert) column: exclusive prefix of the per-block counts over the blocks, in place,
 // and the column total.  A lane owns a contiguous run of blocks, so all its loads are issued at once.
 __global__ void __launch_bounds__(128) group_colscan_kernel(const GroupParams p) {
+  pdl_grid_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int col = blockIdx.x * (blockDim.x >> 5) + warp;
   if (col >= 2 * p.n) return;
@@ -117,9 +119,8 @@ __global__ void __launch_bounds__(128) group_colscan_kernel(const GroupParams p)
 // Offsets over the experts and the 128-row tile schedule of one stage, from the column totals (one warp).
 // Every scatter block computes them for itself; block 0 also publishes them, the statistics, and the
 // padding entries of the stage-1 gather map.
-__device__ __forceinline__ void expert_prefix(const GroupParams &p, int stage, int32_t *offs_s, int32_t *tb_s,
-                                              bool publish, int lane) {
-  const int32_t *cnt = p.col_tot + stage * p.n;
+__device__ __forceinline__ void expert_prefix(const GroupParams &p, int stage, const int32_t *cnt, int32_t *offs_s,
+                                              int32_t *tb_s, bool publish, int lane) {
   int32_t *offs = stage == 0 ? p.g.s1_offsets : p.g.s2_offsets;
   int32_t *tb = stage == 0 ? p.tile_base1 : p.tile_base2;
   int carry_rows = 0, carry_tiles = 0, empty = 0;
@@ -165,8 +166,9 @@ __device__ __forceinline__ int bits_below(const uint32_t *row, int idx) {
   return r + __popc(row[word] & ((1u << (idx & 31)) - 1u));
 }
 
-__global__ void group_scatter_kernel(const GroupParams p) {
-  extern __shared__ int32_t sm[];
+// Body of the scatter step for one block.  `cnt` = rows per (stage, expert) over the whole batch; `single` = the
+// batch is this one block (its per-block offsets are zero).
+__device__ __forceinline__ void scatter_block(const GroupParams &p, int32_t *sm, const int32_t *cnt, bool single) {
   const int CK = p.chunk * p.K;
   const int W = (CK + 31) >> 5;
   int32_t *ssrc = sm, *stgt = ssrc + CK, *srow = stgt + CK;
@@ -176,13 +178,13 @@ __global__ void group_scatter_kernel(const GroupParams p) {
 
   for (int x = threadIdx.x; x < 2 * p.n * W; x += blockDim.x) bits1[x] = 0u;
   if (threadIdx.x < 32) {
-    expert_prefix(p, 0, off1, tb1, blockIdx.x == 0, threadIdx.x);
-    expert_prefix(p, 1, off2, tb2, blockIdx.x == 0, threadIdx.x);
+    expert_prefix(p, 0, cnt, off1, tb1, blockIdx.x == 0, threadIdx.x);
+    expert_prefix(p, 1, cnt + p.n, off2, tb2, blockIdx.x == 0, threadIdx.x);
   }
   if (p.nb > 0) {
     for (int e = threadIdx.x; e < p.n; e += blockDim.x) {
-      bo1[e] = p.blk_cnt[(size_t)e * p.nb + blockIdx.x];
-      bo2[e] = p.blk_cnt[(size_t)(p.n + e) * p.nb + blockIdx.x];
+      bo1[e] = single ? 0 : p.blk_cnt[(size_t)e * p.nb + blockIdx.x];
+      bo2[e] = single ? 0 : p.blk_cnt[(size_t)(p.n + e) * p.nb + blockIdx.x];
     }
   }
   const int nt = p.nb > 0 ? stage_chunk(p, ssrc, stgt) : 0;
@@ -238,6 +240,38 @@ __global__ void group_scatter_kernel(const GroupParams p) {
   }
 }
 
+__global__ void group_scatter_kernel(const GroupParams p) {
+  extern __shared__ int32_t sm[];
+  pdl_grid_wait();
+  scatter_block(p, sm, p.col_tot, false);
+}
+
+// A batch that fits one block (decode steps): histogram, offsets and scatter in a single launch.  The block
+// also clears the plan header itself, so no memset precedes it.
+__global__ void group_single_block_kernel(const GroupParams p) {
+  extern __shared__ int32_t sm[];
+  __shared__ int32_t cnt[2 * kMaxExperts];
+  pdl_grid_wait();
+  if (threadIdx.x == 0) p.plan->status = 0;
+  for (int e = threadIdx.x; e < 2 * p.n; e += blockDim.x) cnt[e] = 0;
+  __syncthreads();
+  {
+    int32_t *ssrc = sm, *stgt = sm + p.chunk * p.K;
+    const int nt = stage_chunk(p, ssrc, stgt);
+    __syncthreads();
+    if ((int)threadIdx.x < nt) {
+      const int32_t *rs = ssrc + threadIdx.x * p.K, *rt = stgt + threadIdx.x * p.K;
+      for (int k = 0; k < p.K; ++k) {
+        if (rs[k] < 0) continue;
+        if (first_occurrence(rs, k, p.dedup) == k) atomicAdd(&cnt[rs[k]], 1);
+        atomicAdd(&cnt[p.n + rt[k]], 1);
+      }
+    }
+    __syncthreads();
+  }
+  scatter_block(p, sm, cnt, true);
+}
+
 pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src, const int32_t *tgt,
                             const float *w, const pcomoe_groups *g, char *ws, const WsLayout &lay,
                             cudaStream_t st) {
@@ -255,10 +289,6 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
   p.T = T; p.n = c.n_experts; p.K = c.top_k; p.dedup = c.dedup; p.chunk = group_chunk_for(L, T);
   p.nb = (T + p.chunk - 1) / p.chunk;
 
-  // the status word and the plan start from zero (the scan kernel fills the padding of the gather map)
-  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.plan, 0, sizeof(DevPlan), st));
-  count_launch();
-
   const int CK = p.chunk * p.K, W = (CK + 31) / 32;
   const size_t smem_count = sizeof(int32_t) * ((size_t)2 * CK + 2 * p.n);
   const size_t smem_scatter = sizeof(int32_t) * ((size_t)3 * CK + 6 * p.n + (size_t)2 * p.n * W);
@@ -267,12 +297,19 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(group_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_count));
   if (smem_scatter > 48 * 1024)
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(group_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_scatter));
-  if (p.nb > 0) {
-    group_count_kernel<<<p.nb, p.chunk, smem_count, st>>>(p);
+  if (p.nb <= 1) {   // the whole batch in one block: one launch does everything
+    if (smem_scatter > 48 * 1024)
+      PCOMOE_CUDA_TRY(cudaFuncSetAttribute(group_single_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_scatter));
+    PCOMOE_CUDA_TRY(launch_pdl(group_single_block_kernel, dim3(1), dim3(p.chunk), smem_scatter, st, p));
     count_launch();
+    return PCOMOE_OK;
   }
-  group_colscan_kernel<<<(2 * p.n + 3) / 4, 128, 0, st>>>(p);
-  group_scatter_kernel<<<p.nb > 0 ? p.nb : 1, p.chunk, smem_scatter, st>>>(p);
+  // the status word and the plan start from zero
+  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.plan, 0, sizeof(DevPlan), st));
+  PCOMOE_CUDA_TRY(launch_pdl(group_count_kernel, dim3(p.nb), dim3(p.chunk), smem_count, st, p));
+  count_launch(2);
+  PCOMOE_CUDA_TRY(launch_pdl(group_colscan_kernel, dim3((2 * p.n + 3) / 4), dim3(128), 0, st, p));
+  PCOMOE_CUDA_TRY(launch_pdl(group_scatter_kernel, dim3(p.nb), dim3(p.chunk), smem_scatter, st, p));
   count_launch(2);
   PCOMOE_CUDA_TRY(cudaGetLastError());
   return PCOMOE_OK;

@@ -103,6 +103,7 @@ __device__ __forceinline__ float warp_max(float v) {
 template <int KMAX>
 __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_grid_wait();
   const int warps = blockDim.x >> 5;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float *zrows = reinterpret_cast<float *>(smem_raw);                 // [warps][2][n]
@@ -251,9 +252,8 @@ pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, con
   else kern = route_kernel<32>;
   if (smem > 48 * 1024)
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<grid, threads, smem, st>>>(p);
+  PCOMOE_CUDA_TRY(launch_pdl(kern, dim3(grid), dim3(threads), smem, st, p));
   count_launch();
-  PCOMOE_CUDA_TRY(cudaGetLastError());
   return PCOMOE_OK;
 }
 
