@@ -44,7 +44,7 @@ typedef enum {
 
 typedef enum { PCOMOE_BF16 = 0, PCOMOE_FP32 = 1 } pcomoe_dtype;
 
-/* Which kernels pcomoe_ffn_forward uses. */
+/* Which kernels pcomoe_ffn_forward uses.  Every choice runs on the GPU; there is no host fallback. */
 typedef enum {
   PCOMOE_FFN_AUTO = 0,   /* tensor-core path when dtype and sizes allow (CTA pairs when groups average
                             at least 256 rows, else one CTA per tile), else the SIMT path        */
