@@ -90,6 +90,18 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
                                   const float *h_bias, pcomoe_layer **out);
 pcomoe_status pcomoe_layer_destroy(pcomoe_layer *layer);
 
+/*
+ * Host utility: a compatibility mask from a compatibility bias (Sec. 4.2: the learned bias is turned into a
+ * layer-specific active mask that keeps every diagonal path and filters low-value off-diagonal routes; the
+ * paper gives no criterion, so the reading here is "keep the off-diagonal entries with the largest bias").
+ *   h_bias [n*n] fp32;  keep_fraction in [0,1]: share of the n(n-1) off-diagonal paths that stay active,
+ *   rounded to the nearest count; ties are broken by the smaller flat id i*n+j.  h_mask [n*n] uint8 receives
+ *   m_ii = 1 and m_ij = 1 for the kept pairs.  Pure host code; tightening the mask over a schedule is calling
+ *   this with a decreasing keep_fraction.
+ * Errors: INVALID_ARG (NULL, n <= 0, keep_fraction outside [0,1] or not finite).
+ */
+pcomoe_status pcomoe_mask_from_bias(int32_t n, const float *h_bias, float keep_fraction, uint8_t *h_mask);
+
 /* Number of active paths |A| of the layer; copies up to `cap` table entries to host arrays
  * (any of them may be NULL).  For checking the table against the mask. */
 pcomoe_status pcomoe_layer_active_set(const pcomoe_layer *layer, int32_t cap, int32_t *h_src,

@@ -61,6 +61,16 @@ def active_set(mask, bias):
     return src[:cnt].copy(), tgt[:cnt].copy(), b[:cnt].copy()
 
 
+def mask_from_bias(bias, keep: int):
+    b = _c(bias, np.float32)
+    n = b.shape[0]
+    m = np.zeros((n, n), np.uint8)
+    rc = _load().pcomoe_oracle_mask_from_bias(ctypes.c_int32(n), _p(b), ctypes.c_int64(keep), _p(m))
+    if rc != 0:
+        raise ValueError(f"pcomoe_oracle_mask_from_bias failed with code {rc}")
+    return m
+
+
 def route(logits, mask, bias, lam, K, tgt_logits=None, norm_topk=1, routed_scale=1.0, with_scores=False):
     z = _c(logits, np.float32)
     u = z if tgt_logits is None else _c(tgt_logits, np.float32)

@@ -331,3 +331,23 @@ int pcomoe_oracle_ffn_grouped(int32_t T, int32_t H, int32_t F, int32_t n, const 
   free(hd);
   return ORACLE_OK;
 }
+
+/* ---------------------------------------------------------------------------
+ * Mask from bias (Sec. 4.2: the bias is converted into an active mask with m_ii = 1 that filters low-value
+ * off-diagonal routes; the criterion is not given - reading: keep the `keep` off-diagonal pairs with the
+ * largest bias, ties to the smaller flat id).  Selection by repeated arg-max: plain and slow.
+ * ------------------------------------------------------------------------- */
+int pcomoe_oracle_mask_from_bias(int32_t n, const float *B, int64_t keep, uint8_t *M) {
+  if (n <= 0 || keep < 0 || keep > (int64_t)n * (n - 1)) return ORACLE_ERR_ARG;
+  for (int32_t i = 0; i < n * n; ++i) M[i] = 0;
+  for (int32_t i = 0; i < n; ++i) M[(size_t)i * n + i] = 1;
+  for (int64_t r = 0; r < keep; ++r) {
+    int32_t best = -1;
+    for (int32_t p = 0; p < n * n; ++p) {
+      if (p / n == p % n || M[p]) continue;
+      if (best < 0 || B[p] > B[best]) best = p;
+    }
+    M[best] = 1;
+  }
+  return ORACLE_OK;
+}

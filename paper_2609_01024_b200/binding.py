@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_WORKSPACE
 PCOMOE_BF16, PCOMOE_FP32 = 0, 1
 PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR = 0, 1, 2, 3
 
-EXPORTS = ["pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
+EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
            "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",
            "pcomoe_ffn_forward_stages",
            "pcomoe_device_status",
@@ -60,6 +60,7 @@ def load_library(path: str | None = None):
     lib = ctypes.CDLL(p)
     vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
     lib.pcomoe_layer_create.argtypes = [ctypes.POINTER(pcomoe_config), vp, vp, ctypes.POINTER(vp)]
+    lib.pcomoe_mask_from_bias.argtypes = [i32, vp, ctypes.c_float, vp]
     lib.pcomoe_layer_destroy.argtypes = [vp]
     lib.pcomoe_layer_active_set.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(i32)]
     lib.pcomoe_workspace_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
@@ -107,6 +108,16 @@ def pcomoe_layer_create(*, n_experts, top_k, hidden, ffn, mask, bias, shared_ffn
     _check(lib.pcomoe_layer_create(ctypes.byref(cfg), m.ctypes.data_as(ctypes.c_void_p),
                                    b.ctypes.data_as(ctypes.c_void_p), ctypes.byref(out)), "pcomoe_layer_create")
     return out
+
+
+def pcomoe_mask_from_bias(bias, keep_fraction: float) -> np.ndarray:
+    """Host utility: mask that keeps the diagonal and the `keep_fraction` largest-bias off-diagonal paths."""
+    b = np.ascontiguousarray(bias, dtype=np.float32)
+    n = b.shape[0]
+    m = np.zeros((n, n), np.uint8)
+    _check(load_library().pcomoe_mask_from_bias(n, b.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(keep_fraction),
+                                                m.ctypes.data_as(ctypes.c_void_p)), "pcomoe_mask_from_bias")
+    return m
 
 
 def pcomoe_layer_destroy(layer):

@@ -1,5 +1,8 @@
 // Host side of the C ABI: layer set-up, workspace sizing, argument checks and dispatch.
+#include <algorithm>
 #include <atomic>
+#include <cmath>
+#include <vector>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -118,6 +121,22 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
     return PCOMOE_ERR_CUDA;
   }
   *out = L;
+  return PCOMOE_OK;
+}
+
+pcomoe_status pcomoe_mask_from_bias(int32_t n, const float *h_bias, float keep_fraction, uint8_t *h_mask) {
+  if (n <= 0 || !h_bias || !h_mask || !(keep_fraction >= 0.0f && keep_fraction <= 1.0f)) return PCOMOE_ERR_INVALID_ARG;
+  const int64_t off = (int64_t)n * (n - 1);
+  const int64_t keep = (int64_t)std::llround((double)keep_fraction * (double)off);
+  std::vector<int32_t> order;
+  order.reserve((size_t)off);
+  for (int32_t i = 0; i < n; ++i)
+    for (int32_t j = 0; j < n; ++j)
+      if (i != j) order.push_back(i * n + j);
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return h_bias[a] > h_bias[b]; });
+  std::memset(h_mask, 0, (size_t)n * n);
+  for (int32_t i = 0; i < n; ++i) h_mask[(size_t)i * n + i] = 1;
+  for (int64_t r = 0; r < keep; ++r) h_mask[order[(size_t)r]] = 1;
   return PCOMOE_OK;
 }
 
