@@ -753,6 +753,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
         const CUtensorMap *mA = t.seg ? &tmA1 : &tmA0;
         const CUtensorMap *mB;
         int b_row;
+        // a pair half without a tile reads rows far outside the tensor: TMA fills them with zeros
+        const int a_row = t.valid > 0 ? t.prow0 : 0x3fffff80;
         if (STAGE == 1) {            // leader: 128 gate rows; peer: the matching 128 up rows
           mB = rank == 0 ? (t.seg ? &tmB1 : &tmB0) : (t.seg ? &tmC1 : &tmC0);
           b_row = t.g * S.b_group_rows + t.n_idx * 128;
@@ -765,7 +767,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
           const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
           const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
-          tma_load_2d_pair(sa, mA, kb * BK, t.prow0, lead_full);
+          tma_load_2d_pair(sa, mA, kb * BK, a_row, lead_full);
           tma_load_2d_pair(sb, mB, kb * BK, b_row, lead_full);
           if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
         }
@@ -844,22 +846,25 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   }
 }
 
-// Copies rows idx[r] of src into consecutive rows of dst (the A operand of stage 1 in group order).
-// One warp per row; a lane keeps up to eight 16-byte loads in flight before it stores.
+// Copies rows idx[r] of src into consecutive rows of dst (the A operand of stage 1 in group order); a negative
+// index marks a padding row, which is written as zeros (zero operands keep the tensor cores' switching power
+// down for rows whose results are dropped).  One warp per row; up to eight 16-byte loads in flight per lane.
 __global__ void __launch_bounds__(256) gather_rows_kernel(uint4 *dst, const uint4 *src, const int32_t *idx,
                                                           const int32_t *tile_base, int G, int vec_per_row) {
   pdl_grid_wait();
   const int rows = tile_base[G] * kTileM;
   const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
   for (int r = blockIdx.x * warps_per_block + (threadIdx.x >> 5); r < rows; r += gridDim.x * warps_per_block) {
-    const uint4 *s = src + (size_t)idx[r] * vec_per_row;
+    const int tok = idx[r];
+    const uint4 *s = src + (size_t)(tok < 0 ? 0 : tok) * vec_per_row;
     uint4 *d = dst + (size_t)r * vec_per_row;
     for (int v0 = 0; v0 < vec_per_row; v0 += 256) {
       uint4 x[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int v = v0 + i * 32 + lane;
-        if (v < vec_per_row) x[i] = __ldg(s + v);
+        x[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (v < vec_per_row && tok >= 0) x[i] = __ldg(s + v);
       }
 #pragma unroll
       for (int i = 0; i < 8; ++i) {

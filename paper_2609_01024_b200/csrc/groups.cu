@@ -136,8 +136,8 @@ __device__ __forceinline__ void expert_prefix(const GroupParams &p, int stage, c
       if (publish) {
         offs[e] = o;
         tb[e] = t0;
-        if (stage == 0)  // the padding rows of a source group gather token 0 (any valid row will do)
-          for (int x = c; x < tl * kTileM; ++x) p.a1_idx[(size_t)t0 * kTileM + x] = 0;
+        if (stage == 0)  // the padding rows of a source group have no token: they are gathered as zeros
+          for (int x = c; x < tl * kTileM; ++x) p.a1_idx[(size_t)t0 * kTileM + x] = -1;
       }
     }
     empty += __popc(__ballot_sync(0xffffffffu, e < p.n && c == 0));
