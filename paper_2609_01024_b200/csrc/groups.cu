@@ -136,8 +136,6 @@ __device__ __forceinline__ void expert_prefix(const GroupParams &p, int stage, c
       if (publish) {
         offs[e] = o;
         tb[e] = t0;
-        if (stage == 0)  // the padding rows of a source group have no token: they are gathered as zeros
-          for (int x = c; x < tl * kTileM; ++x) p.a1_idx[(size_t)t0 * kTileM + x] = -1;
       }
     }
     empty += __popc(__ballot_sync(0xffffffffu, e < p.n && c == 0));
@@ -189,6 +187,14 @@ __device__ __forceinline__ void scatter_block(const GroupParams &p, int32_t *sm,
   }
   const int nt = p.nb > 0 ? stage_chunk(p, ssrc, stgt) : 0;
   __syncthreads();
+
+  // the padding rows of the source groups have no token: they are gathered as zeros (marked -1).  The blocks
+  // share the groups among themselves.
+  for (int e = blockIdx.x; e < p.n; e += gridDim.x) {
+    const int c = cnt[e];
+    const int rows = (c + kTileM - 1) / kTileM * kTileM;
+    for (int x = c + threadIdx.x; x < rows; x += blockDim.x) p.a1_idx[(size_t)tb1[e] * kTileM + x] = -1;
+  }
 
   const int tl = threadIdx.x;
   const int32_t *rs = ssrc + tl * p.K, *rt = stgt + tl * p.K;
