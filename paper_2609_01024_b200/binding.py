@@ -303,6 +303,49 @@ class PathMoELayer:
         torch.cuda.current_stream().synchronize()
         return self._pin_y[:T].numpy()
 
+    def stream_from_host(self, pinned_logits, pinned_h, steps: int):
+        """Serving loop over `steps` batches that live in PINNED host memory (torch CPU tensors; `pinned_h` is
+        bf16 or fp32).  Every step copies its inputs host->device, runs the hot path and copies y device->host;
+        the three are put on separate streams with two buffer slots, so the copies of neighbouring steps
+        overlap the kernels.  Returns the pinned y of the last step (synchronised).  Marshalling only."""
+        T = pinned_h.shape[0]
+        assert pinned_logits.is_pinned() and pinned_h.is_pinned() and T <= self.max_tokens
+        if getattr(self, "_slots", None) is None or self._slots["T"] < T:
+            mk = lambda *shape, dtype: [torch.empty(*shape, dtype=dtype, device=self.device) for _ in range(2)]
+            self._slots = dict(T=T, logits=mk(T, self.n, dtype=torch.float32), h=mk(T, self.H, dtype=pinned_h.dtype),
+                               y=mk(T, self.H, dtype=torch.float32),
+                               out=[torch.empty(T, self.H, dtype=torch.float32).pin_memory() for _ in range(2)],
+                               s_in=torch.cuda.Stream(self.device), s_out=torch.cuda.Stream(self.device))
+        sl = self._slots
+        main = torch.cuda.current_stream()
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_done = [torch.cuda.Event() for _ in range(2)]     # kernels of the slot finished (inputs free, y ready)
+        ev_out = [torch.cuda.Event() for _ in range(2)]      # y of the slot copied out (y buffer free)
+        y_keep = self.y
+        for i in range(steps):
+            s = i & 1
+            with torch.cuda.stream(sl["s_in"]):
+                if i >= 2:
+                    sl["s_in"].wait_event(ev_done[s])
+                sl["logits"][s][:T].copy_(pinned_logits[:T], non_blocking=True)
+                sl["h"][s][:T].copy_(pinned_h[:T], non_blocking=True)
+                ev_in[s].record(sl["s_in"])
+            main.wait_event(ev_in[s])
+            if i >= 2:
+                main.wait_event(ev_out[s])
+            self.y = sl["y"][s]
+            self.forward(sl["logits"][s][:T], sl["h"][s][:T])
+            ev_done[s].record(main)
+            with torch.cuda.stream(sl["s_out"]):
+                sl["s_out"].wait_event(ev_done[s])
+                sl["out"][s][:T].copy_(sl["y"][s][:T], non_blocking=True)
+                ev_out[s].record(sl["s_out"])
+        self.y = y_keep
+        last = (steps - 1) & 1
+        ev_out[last].synchronize()
+        main.synchronize()
+        return sl["out"][last][:T]
+
     def device_status(self) -> int:
         return pcomoe_device_status(self.workspace)
 

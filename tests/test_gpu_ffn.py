@@ -120,3 +120,20 @@ def test_vanilla_reduction_on_gpu(G, oracle):
     assert np.array_equal(layer.path_src[:cfg.T].cpu().numpy(), idx)
     assert np.array_equal(layer.path_tgt[:cfg.T].cpu().numpy(), idx)
     G.check_output(y, yv)
+
+
+def test_streaming_from_pinned_host_buffers(G, oracle):
+    """The overlapped serving loop (copies and kernels on separate streams, two slots) returns the same y."""
+    import torch
+    cfg = wl.small_case(29, T=300, H=256, F=128, n=5, K=2, F_sh=128)
+    L = wl.make_layer(cfg)
+    layer = G.make_gpu_layer(cfg, L)
+    pin_logits = torch.from_numpy(L.logits).pin_memory()
+    pin_h = torch.from_numpy(L.h.view(np.int16)).view(torch.bfloat16).pin_memory()
+    rs, rt, rw = oracle.route(L.logits, L.mask, L.bias, cfg.lam, cfg.K)
+    yr = oracle.ffn(wl.hidden_as_f32(cfg, L.h), L.w_gate, L.w_up, L.w_down, rs, rt, rw,
+                    shared=(L.wsh_gate, L.wsh_up, L.wsh_down))
+    for steps in (1, 2, 5):
+        y = layer.stream_from_host(pin_logits, pin_h, steps).numpy().copy()
+        assert layer.device_status() == 0
+        G.check_output(y, yr)
