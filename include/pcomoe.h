@@ -51,10 +51,8 @@ typedef enum {
   PCOMOE_FFN_SIMT = 1,   /* plain-FMA kernels (any size, bf16 or fp32 storage)               */
   PCOMOE_FFN_TCGEN05 = 2, /* tcgen05 / TMEM / TMA kernels, one CTA per 128 x 256 tile;
                              PCOMOE_ERR_UNSUPPORTED if not bf16 or if H % 256 != 0 or F % 128 != 0 */
-  PCOMOE_FFN_TCGEN05_PAIR = 3, /* the same with two CTAs (a cluster of 2 SMs) per 256 x 256 tile,
-                                  tcgen05.mma.cta_group::2; same size rules                        */
-  PCOMOE_FFN_TCGEN05_SWAP = 4  /* CTA pairs with the weight rows on the M side of the MMA and a block of up
-                                  to 256 token rows on the N side (short last blocks cost less)     */
+  PCOMOE_FFN_TCGEN05_PAIR = 3 /* the same with two CTAs (a cluster of 2 SMs) per 256 x 256 tile,
+                                 tcgen05.mma.cta_group::2; same size rules                        */
 } pcomoe_ffn_impl;
 
 /* Plain data; set struct_size = sizeof(pcomoe_config). */

@@ -18,7 +18,7 @@ PCOMOE_OK = 0
 STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_WORKSPACE", 4: "ERR_UNSUPPORTED",
                 5: "ERR_CUDA", 6: "ERR_TIMEOUT", 7: "ERR_INDEX"}
 PCOMOE_BF16, PCOMOE_FP32 = 0, 1
-PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR, PCOMOE_FFN_TCGEN05_SWAP = 0, 1, 2, 3, 4
+PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR = 0, 1, 2, 3
 
 EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
            "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",

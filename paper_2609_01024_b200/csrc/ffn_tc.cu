@@ -846,473 +846,6 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   }
 }
 
-// =====================================================================================================
-// Weights-on-M variant ("swap").  The CTA pair's 256 MMA rows are WEIGHT rows and the N dimension is a block of up
-// to 256 token rows of one group, so the last, short block of a group costs MMA time in proportion to its rows
-// (N is rounded up to 32) instead of a whole tile.  Per pair tile: stage 1 = 128 intermediate columns (each CTA:
-// 64 gate rows in TMEM lanes 0-63 and the 64 matching up rows in lanes 64-127) x one token block; stage 2 = 256
-// output columns (128 per CTA) x one block of path rows.  Accumulators are transposed: lane = weight row,
-// column = token.  Stage-1 epilogue: the up half hands its values to the gate half through shared memory,
-// SiLU(g)*u is written token-major into shared memory, and every token row leaves as 128 contiguous bytes to each
-// stage-2 row that reuses it.  Stage-2 epilogue: for each token column a warp adds 32 consecutive floats of
-// y[token] (one whole line per instruction), scaled by the path weight.
-// =====================================================================================================
-constexpr int kSwapDst = 4;
-constexpr uint32_t kIdescSwapBase = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 4) << 24);   // M = 256, N at run time
-
-struct SwapTile {
-  int seg, g, n_idx;
-  int prow0;    // first padded row of the token block
-  int urow0;    // first unpadded row of the token block
-  int valid;    // rows of the block that exist (1..256)
-  int npad;     // valid rounded up to a multiple of 32: the N of the MMAs
-};
-
-struct SwapWalker {
-  const int32_t *tb, *ro, *pb;   // [2][kMaxExperts + 2] each: m-tile prefix, row offsets, token-block prefix
-  int nt[2], G[2], nseg;
-  int seg, g, seg_first;
-  __device__ int seg_tiles(int s) const { return pb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
-  __device__ int total() const {
-    int t = 0;
-    for (int s = 0; s < nseg; ++s) t += seg_tiles(s);
-    return t;
-  }
-  __device__ SwapTile at(int tile) {
-    while (seg + 1 < nseg && tile >= seg_first + seg_tiles(seg)) {
-      seg_first += seg_tiles(seg);
-      ++seg;
-      g = 0;
-    }
-    const int o = seg * (kMaxExperts + 2);
-    const int32_t *b = tb + o, *r = ro + o, *q = pb + o;
-    const int n_t = nt[seg], local_seg = tile - seg_first;
-    while (g + 1 < G[seg] && local_seg >= q[g + 1] * n_t) ++g;
-    SwapTile t;
-    const int nblk = q[g + 1] - q[g];
-    const int local = local_seg - q[g] * n_t;
-    t.seg = seg;
-    t.g = g;
-    t.n_idx = local / nblk;
-    const int blk = local - t.n_idx * nblk;
-    t.prow0 = (b[g] + 2 * blk) * kTileM;
-    t.urow0 = r[g] + 2 * blk * kTileM;
-    t.valid = min(2 * kTileM, r[g + 1] - t.urow0);
-    t.npad = max(32, (t.valid + 31) & ~31);
-    return t;
-  }
-};
-
-__device__ __forceinline__ void umma_bf16_pair_n(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                                 uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the 4 epilogue warps
-// barrier of the 4 epilogue warps that also tells every thread whether any of them raised `flag`
-__device__ __forceinline__ bool epi_any(bool flag) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 p, %1, 0;\n\t"
-      "bar.red.or.pred q, 1, 128, p;\n\t"
-      "selp.u32 %0, 1, 0, q;\n\t}"
-      : "=r"(r)
-      : "r"((uint32_t)flag)
-      : "memory");
-  return r != 0;
-}
-__device__ __forceinline__ void red_add_f32(float *addr, float v) {
-  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
-}
-
-// ---- epilogues of a weights-on-M block (TMEM lane = weight row, column = token row); they return false when the
-// ---- CTA is giving up.  Called by the four epilogue warps together; they start and end with a barrier of those
-// ---- warps, so the shared buffers never overlap the per-warp staging of a neighbouring ordinary tile.
-__device__ __forceinline__ bool swap_epilogue_stage2(const TcParams &p, const Seg &S, const SwapTile &t, uint32_t rank,
-                                                     int quarter, int lane, int et, uint32_t taddr, uint32_t accf,
-                                                     uint32_t acc_phase, volatile int *abort_flag, int32_t *s_dst) {
-  const int nchunks = t.npad >> 5;
-  int2 *tw = reinterpret_cast<int2 *>(s_dst);
-  // (token, weight) of every row of the block
-  for (int j = et; j < t.npad; j += 128) {
-    int tok = -1;
-    float w = 0.0f;
-    if (j < t.valid) {
-      const int urow = t.urow0 + j;
-      tok = S.s2_token ? S.s2_token[urow] : urow;
-      w = S.s2_w ? S.s2_w[urow] : 1.0f;
-      if ((unsigned)tok >= (unsigned)p.T) {
-        atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
-        tok = -1;
-      }
-    }
-    tw[j] = make_int2(tok, __float_as_int(w));
-  }
-  // the give-up decision is shared by the four warps (nobody may be left alone at a later barrier); the
-  // same barrier publishes the table
-  if (epi_any(!mbar_wait(accf, acc_phase, abort_flag))) return false;
-  tc_fence_after();
-  float *ycol = p.y + (size_t)t.n_idx * 256 + rank * 128 + quarter * 32 + lane;
-  uint32_t v0[32], v1[32];
-  tmem_ld32_issue(taddr, v0);
-  for (int c = 0; c < nchunks; c += 2) {
-    tmem_wait_ld();
-    reg_fence32(v0);
-    if (c + 1 < nchunks) tmem_ld32_issue(taddr + (c + 1) * 32, v1);
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-      const int2 e = tw[c * 32 + j];
-      if (e.x >= 0) red_add_f32(ycol + (size_t)e.x * p.ldy, __int_as_float(e.y) * __uint_as_float(v0[j]));
-    }
-    if (c + 1 < nchunks) {
-      tmem_wait_ld();
-      reg_fence32(v1);
-      if (c + 2 < nchunks) tmem_ld32_issue(taddr + (c + 2) * 32, v0);
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int2 e = tw[(c + 1) * 32 + j];
-        if (e.x >= 0) red_add_f32(ycol + (size_t)e.x * p.ldy, __int_as_float(e.y) * __uint_as_float(v1[j]));
-      }
-    }
-  }
-  return true;
-}
-
-__device__ __forceinline__ bool swap_epilogue_stage1(const TcParams &p, const Seg &S, const SwapTile &t, uint32_t rank,
-                                                     int quarter, int lane, int et, int wq, uint32_t taddr,
-                                                     uint32_t accf, uint32_t acc_phase, volatile int *abort_flag,
-                                                     uint32_t *s_epi, int32_t *s_dst, uint32_t &obuf_sel) {
-  const int nchunks = t.npad >> 5;
-  float *ubuf = reinterpret_cast<float *>(s_epi);                           // [64][kEpiStride]
-  uint32_t *obuf0 = s_epi + 64 * kEpiStride;                                // 2 x [32][kEpiStride words]
-  const bool up_half = quarter >= 2;
-  const int frow = (quarter & 1) * 32 + lane;                               // 0..63 within the half
-  const size_t col0 = (size_t)t.n_idx * 128 + rank * 64;                    // first output column of this CTA
-  // where every token row of the block goes (looked up while the MMAs of the block run)
-  for (int row = et; row < t.npad; row += 128) {
-    int d[kSwapDst];
-#pragma unroll
-    for (int j = 0; j < kSwapDst; ++j) d[j] = -1;
-    if (row < t.valid) {
-      const int prow = t.prow0 + row;
-      if (!S.row_token) {
-        d[0] = prow;
-      } else {
-        const int tok = S.row_token[prow];
-        if ((unsigned)tok >= (unsigned)p.T) {
-          atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
-        } else {
-          int nd = 0;
-          for (int k = 0; k < p.K; ++k) {
-            if (S.path_prow1[(size_t)tok * p.K + k] != prow) continue;
-            const int x = S.path_pos2[(size_t)tok * p.K + k];
-#pragma unroll
-            for (int j = 0; j < kSwapDst; ++j)
-              if (j == nd) d[j] = x;
-            ++nd;
-          }
-          if (nd > kSwapDst) d[0] = -2;
-        }
-      }
-    }
-    *reinterpret_cast<int4 *>(s_dst + row * kSwapDst) = make_int4(d[0], d[1], d[2], d[3]);
-  }
-  if (epi_any(!mbar_wait(accf, acc_phase, abort_flag))) return false;
-  tc_fence_after();
-  uint32_t va[32], vb[32];
-  tmem_ld32_issue(taddr, va);
-  auto chunk = [&](int c, uint32_t (&v)[32]) {
-    if (up_half) {
-#pragma unroll
-      for (int q = 0; q < 8; ++q)
-        *reinterpret_cast<uint4 *>(ubuf + frow * kEpiStride + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-    }
-    epi_barrier();
-    uint32_t *obuf = obuf0 + (obuf_sel & 1u) * (32 * kEpiStride);
-    if (!up_half) {
-      __nv_bfloat16 *ob = reinterpret_cast<__nv_bfloat16 *>(obuf) + frow;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        const float4 u4 = *reinterpret_cast<const float4 *>(ubuf + frow * kEpiStride + 4 * q);
-        ob[(4 * q) * (kEpiStride * 2)] = __float2bfloat16_rn(silu_mul(__uint_as_float(v[4 * q]), u4.x));
-        ob[(4 * q + 1) * (kEpiStride * 2)] = __float2bfloat16_rn(silu_mul(__uint_as_float(v[4 * q + 1]), u4.y));
-        ob[(4 * q + 2) * (kEpiStride * 2)] = __float2bfloat16_rn(silu_mul(__uint_as_float(v[4 * q + 2]), u4.z));
-        ob[(4 * q + 3) * (kEpiStride * 2)] = __float2bfloat16_rn(silu_mul(__uint_as_float(v[4 * q + 3]), u4.w));
-      }
-    }
-    epi_barrier();
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int r = wq * 8 + i * 4 + (lane >> 3);               // token row within the chunk
-      const int4 d = *reinterpret_cast<const int4 *>(s_dst + (c * 32 + r) * kSwapDst);
-      const uint4 x = *reinterpret_cast<const uint4 *>(obuf + r * kEpiStride + (lane & 7) * 4);
-      __nv_bfloat16 *out_col = S.u_out + col0 + (lane & 7) * 8;
-      if (d.x >= 0) {
-        *reinterpret_cast<uint4 *>(out_col + (size_t)d.x * S.ldu) = x;
-        if (d.y >= 0) *reinterpret_cast<uint4 *>(out_col + (size_t)d.y * S.ldu) = x;
-        if (d.z >= 0) *reinterpret_cast<uint4 *>(out_col + (size_t)d.z * S.ldu) = x;
-        if (d.w >= 0) *reinterpret_cast<uint4 *>(out_col + (size_t)d.w * S.ldu) = x;
-      } else if (d.x == -2) {
-        const int prow = t.prow0 + c * 32 + r;
-        const int tok = S.row_token[prow];
-        for (int k = 0; k < p.K; ++k)
-          if (S.path_prow1[(size_t)tok * p.K + k] == prow)
-            *reinterpret_cast<uint4 *>(out_col + (size_t)S.path_pos2[(size_t)tok * p.K + k] * S.ldu) = x;
-      }
-    }
-    ++obuf_sel;
-  };
-  for (int c = 0; c < nchunks; c += 2) {
-    tmem_wait_ld();
-    reg_fence32(va);
-    if (c + 1 < nchunks) tmem_ld32_issue(taddr + (c + 1) * 32, vb);
-    chunk(c, va);
-    if (c + 1 < nchunks) {
-      tmem_wait_ld();
-      reg_fence32(vb);
-      if (c + 2 < nchunks) tmem_ld32_issue(taddr + (c + 2) * 32, va);
-      chunk(c + 1, vb);
-    }
-  }
-  return true;
-}
-
-// Pair tiles of the mixed kernel: whole pairs of 128-row m-tiles are ordinary 256 x 256 tiles; the odd last m-tile of
-// a group becomes a weights-on-M block (sw.npad > 0) whose MMA time follows its row count.
-struct MixWalker : PairWalker {
-  __device__ TileInfo at(int tile, int rank, SwapTile &sw) {
-    TileInfo t = PairWalker::at(tile, rank);
-    const int o = seg * (kMaxExperts + 2);
-    const int32_t *b = tb + o, *r = ro + o;
-    const int mt = b[g + 1] - b[g], m0 = t.m_idx - rank;
-    sw.npad = 0;
-    if (m0 + 1 >= mt) {   // no second m-tile: the block has at most 128 rows
-      sw.seg = t.seg; sw.g = t.g; sw.n_idx = t.n_idx;
-      sw.prow0 = (b[g] + m0) * kTileM;
-      sw.urow0 = r[g] + m0 * kTileM;
-      sw.valid = r[g + 1] - sw.urow0;
-      sw.npad = max(32, (sw.valid + 31) & ~31);
-    }
-    return t;
-  }
-};
-
-template <int STAGE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-grouped_gemm_mixed_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
-                         const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
-                         const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmC1,
-                         const __grid_constant__ CUtensorMap tmG0, const __grid_constant__ CUtensorMap tmU0,
-                         const __grid_constant__ CUtensorMap tmG1, const __grid_constant__ CUtensorMap tmU1,
-                         const TcParams p) {
-  extern __shared__ unsigned char smem_dyn[];
-  pdl_grid_wait();
-  __shared__ int32_t s_tb[2 * (kMaxExperts + 2)], s_ro[2 * (kMaxExperts + 2)], s_pb[2 * (kMaxExperts + 2)];
-  __shared__ __align__(8) uint64_t s_bar[2 * STAGES2 + 4];
-  __shared__ uint32_t s_tmem;
-  __shared__ int s_abort;
-  __shared__ __align__(16) float s_epi[4 * 32 * kEpiStride];   // per epilogue warp: 32 rows being turned around
-  __shared__ __align__(16) int32_t s_dst[128 * kSwapDst];      // weights-on-M blocks: readers of each token row / (token, weight)
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
-  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-  const uint32_t bar0 = smem_u32(s_bar);
-  auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES2 + s); };
-  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + a); };
-  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + 2 + a); };
-
-  for (int sg = 0; sg < p.nseg; ++sg) {
-    const Seg &S = p.seg[sg];
-    int32_t *tb = s_tb + sg * (kMaxExperts + 2), *ro = s_ro + sg * (kMaxExperts + 2);
-    if (S.tile_base) {
-      for (int i = threadIdx.x; i <= S.G; i += blockDim.x) {
-        tb[i] = S.tile_base[i];
-        ro[i] = S.row_offsets[i];
-      }
-    } else if (threadIdx.x == 0) {
-      tb[0] = 0; tb[1] = (S.single_rows + kTileM - 1) / kTileM;
-      ro[0] = 0; ro[1] = S.single_rows;
-    }
-  }
-  if (threadIdx.x == 0) {
-    s_abort = 0;
-    for (int s = 0; s < STAGES2; ++s) {
-      mbar_init(full_bar(s), 1);      // the leader's expect_tx arrival; bytes come from both CTAs
-      mbar_init(empty_bar(s), 1);     // one commit (broadcast to both CTAs)
-    }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(accf_bar(a), 1);      // one commit (broadcast)
-      mbar_init(acce_bar(a), 256);    // the epilogue threads of both CTAs
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-  if (warp == 0 && lane < p.nseg) {   // pair prefix per group: ceil(m-tiles / 2)
-    const int sg = lane, o = sg * (kMaxExperts + 2);
-    const int G = p.seg[sg].tile_base ? p.seg[sg].G : 1;
-    int acc = 0;
-    for (int g = 0; g < G; ++g) {
-      s_pb[o + g] = acc;
-      acc += (s_tb[o + g + 1] - s_tb[o + g] + 1) >> 1;
-    }
-    s_pb[o + G] = acc;
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();                 // both CTAs' barriers exist before anything is signalled across
-  tc_fence_after();
-  const uint32_t tmem_base = s_tmem;
-  volatile int *abort_flag = &s_abort;
-
-  MixWalker walk;
-  walk.tb = s_tb; walk.ro = s_ro; walk.pb = s_pb; walk.nseg = p.nseg;
-  for (int sg = 0; sg < 2; ++sg) {
-    walk.nt[sg] = p.seg[sg].nt;
-    walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
-  }
-  walk.seg = 0; walk.g = 0; walk.seg_first = 0;
-  const int total = walk.total();
-
-  if (warp == 0) {
-    // ---------------- producer (both CTAs): own A rows and own half of B ----------------
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      bool alive = true;
-      for (int tile = pair_id; tile < total && alive; tile += n_pairs) {
-        SwapTile sw;
-        const TileInfo t = walk.at(tile, rank, sw);
-        const bool swapped = sw.npad > 0;
-        const Seg &S = p.seg[t.seg];
-        const CUtensorMap *mA = t.seg ? &tmA1 : &tmA0;
-        const CUtensorMap *mB;
-        int b_row;
-        // ordinary tile: this CTA's 128 token rows; weights-on-M block: this CTA's half of the block's N rows
-        const int a_row = swapped ? sw.prow0 + (int)rank * (sw.npad >> 1) : t.prow0;
-        if (STAGE == 1) {            // leader: 128 gate rows; peer: the matching 128 up rows
-          mB = rank == 0 ? (t.seg ? &tmB1 : &tmB0) : (t.seg ? &tmC1 : &tmC0);
-          b_row = t.g * S.b_group_rows + t.n_idx * 128;
-        } else {                     // halves of a 256-row slice of W_down
-          mB = t.seg ? &tmB1 : &tmB0;
-          b_row = t.g * S.b_group_rows + t.n_idx * 256 + (int)rank * 128;
-        }
-        for (int kb = 0; kb < S.kb; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { alive = false; break; }
-          const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
-          const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
-          tma_load_2d_pair(sa, mA, kb * BK, a_row, lead_full);
-          if (STAGE == 1 && swapped) {   // 64 gate rows and the 64 matching up rows of this CTA's 64 columns
-            const int w_row = t.g * S.b_group_rows + t.n_idx * 128 + (int)rank * 64;
-            tma_load_2d_pair(sb, t.seg ? &tmG1 : &tmG0, kb * BK, w_row, lead_full);
-            tma_load_2d_pair(sb + HALF_BYTES / 2, t.seg ? &tmU1 : &tmU0, kb * BK, w_row, lead_full);
-          } else {
-            tma_load_2d_pair(sb, mB, kb * BK, b_row, lead_full);
-          }
-          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ---------------- MMA issuer (leader only) ----------------
-    if (lane == 0 && rank == 0) {
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
-      bool alive = true;
-      for (int tile = pair_id; tile < total && alive; tile += n_pairs) {
-        SwapTile sw;
-        const TileInfo t = walk.at(tile, 0, sw);
-        const bool swapped = sw.npad > 0;
-        const uint32_t idesc = swapped ? (kIdescSwapBase | ((uint32_t)(sw.npad >> 3) << 17)) : kIdescPair;
-        const int nkb = p.seg[t.seg].kb;
-        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
-          tc_fence_after();
-          const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
-          const uint64_t da = umma_desc(sa), db = umma_desc(sb);
-#pragma unroll
-          for (int k = 0; k < BK / 16; ++k)   // weights-on-M blocks take the weight half as the M operand
-            umma_bf16_pair_n(d_tmem, (swapped ? db : da) + 2u * k, (swapped ? da : db) + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          umma_commit_pair(empty_bar(stage));
-          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
-        }
-        if (!alive) break;
-        umma_commit_pair(accf_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-      }
-    }
-    __syncwarp();
-  } else {
-    // ---------------- epilogue (both CTAs, own 128 rows) ----------------
-    const int quarter = warp & 3;
-    const int r = quarter * 32 + lane;
-    if (STAGE == 1 && p.zero_vec4 > 0) {
-      const int et = (warp - 2) * 32 + lane;
-      const int64_t per = (p.zero_vec4 + gridDim.x - 1) / gridDim.x;
-      const int64_t lo = per * blockIdx.x, hi = min(p.zero_vec4, lo + per);
-      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int64_t i = lo + et; i < hi; i += 128) p.zero_ptr[i] = z;
-    }
-    int acc = 0;
-    uint32_t acc_phase = 0, obuf_sel = 0;
-    for (int tile = pair_id; tile < total; tile += n_pairs) {
-      SwapTile sw;
-      const TileInfo t = walk.at(tile, rank, sw);
-      const Seg &S = p.seg[t.seg];
-      const uint32_t taddr = tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16);
-      if (sw.npad > 0) {
-        const int et = (warp - 2) * 32 + lane;
-        const bool ok = STAGE == 1
-            ? swap_epilogue_stage1(p, S, sw, rank, quarter, lane, et, warp - 2, taddr, accf_bar(acc), acc_phase, abort_flag,
-                                   reinterpret_cast<uint32_t *>(s_epi), s_dst, obuf_sel)
-            : swap_epilogue_stage2(p, S, sw, rank, quarter, lane, et, taddr, accf_bar(acc), acc_phase, abort_flag, s_dst);
-        if (!ok) break;
-      } else {
-        const RowCtx c = prepare_row<STAGE>(p, S, t, r);
-        if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
-        tc_fence_after();
-        epilogue_tile<STAGE>(p, S, t, c, taddr, s_epi + (warp - 2) * 32 * kEpiStride);
-      }
-      tc_fence_before();
-      mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));   // the leader's MMA waits for both halves
-      if (sw.npad > 0) epi_barrier();                       // the shared buffers are free again
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-    }
-  }
-
-  // ---------------- teardown ----------------
-  tc_fence_before();
-  __syncthreads();
-  if (s_abort) {
-    if (threadIdx.x == 0) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_TIMEOUT);
-    const uint64_t t0 = global_ns();
-    for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
-  }
-  cluster_sync_all();                 // no signal may reach a CTA that has already exited
-  if (warp == 1) {
-    __syncwarp();
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-  }
-}
-
 // Copies rows idx[r] of src into consecutive rows of dst (the A operand of stage 1 in group order); a negative
 // index marks a padding row, which is written as zeros (zero operands keep the tensor cores' switching power
 // down for rows whose results are dropped).  One warp per row; up to eight 16-byte loads in flight per lane.
@@ -1403,20 +936,17 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
-    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_mixed_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
-    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_mixed_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     attr_done = true;
   }
   // CTA pairs pay off once groups are a few tiles long; short groups (decode) leave the peer CTA idle
-  const bool mixed = c.ffn_impl == PCOMOE_FFN_TCGEN05_SWAP;
-  const bool pair = mixed || c.ffn_impl == PCOMOE_FFN_TCGEN05_PAIR ||
+  const bool pair = c.ffn_impl == PCOMOE_FFN_TCGEN05_PAIR ||
                     (c.ffn_impl == PCOMOE_FFN_AUTO && (int64_t)T * c.top_k >= (int64_t)256 * n);
   const int grid = pair ? (L->sm_count & ~1) : L->sm_count;
   const uint32_t down_box = pair ? 128 : 256;   // a CTA of a pair loads half of the 256-row slice of W_down
 
   // ---- stage 1: rows of h gathered into group order, then one launch over routed + shared tiles ----
   if (stages & (kStage1Routed | kStage1Shared)) {
-    CUtensorMap mA[2], mB[2], mC[2], mG[2], mU[2];   // mG/mU: 64-row boxes of gate/up for weights-on-M blocks
+    CUtensorMap mA[2], mB[2], mC[2];
     TcParams p{};
     p.K = c.top_k; p.T = T; p.plan = plan; p.y = y; p.ldy = H;
     int ns = 0;
@@ -1426,31 +956,26 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
                                  reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8));
       count_launch();
       ok = ok && make_map(&mA[ns], Hg, pad_rows, H, kTileM) && make_map(&mB[ns], wg, (uint64_t)n * F, H, 128) &&
-           make_map(&mC[ns], wu, (uint64_t)n * F, H, 128) && make_map(&mG[ns], wg, (uint64_t)n * F, H, 64) &&
-           make_map(&mU[ns], wu, (uint64_t)n * F, H, 64);
+           make_map(&mC[ns], wu, (uint64_t)n * F, H, 128);
       Seg &S = p.seg[ns++];
       S.tile_base = tb1; S.row_offsets = g->s1_offsets; S.G = n; S.nt = F / 128; S.kb = H / BK; S.b_group_rows = F;
       S.row_token = a1; S.path_prow1 = prow1; S.path_pos2 = pos2; S.u_out = U; S.ldu = F;
     }
     if (stages & kStage1Shared) {
       ok = ok && make_map(&mA[ns], h, (uint64_t)T, H, kTileM) && make_map(&mB[ns], sg, Fsh, H, 128) &&
-           make_map(&mC[ns], su, Fsh, H, 128) && make_map(&mG[ns], sg, Fsh, H, 64) && make_map(&mU[ns], su, Fsh, H, 64);
+           make_map(&mC[ns], su, Fsh, H, 128);
       Seg &S = p.seg[ns++];
       S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
     }
     if (!ok) return PCOMOE_ERR_CUDA;
-    if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; mC[1] = mC[0]; mG[1] = mG[0]; mU[1] = mU[0]; }
+    if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; mC[1] = mC[0]; }
     p.nseg = ns;
     if (stages & kStage2Routed) {   // a full forward: y is cleared here, under the first tile's MMAs
       p.zero_ptr = reinterpret_cast<float4 *>(y);
       p.zero_vec4 = (int64_t)T * H / 4;
     }
-    if (mixed)
-      PCOMOE_CUDA_TRY(launch_pdl(grouped_gemm_mixed_kernel<1>, dim3(grid), dim3(kThreads), kSmemDyn, st, mA[0], mB[0], mC[0],
-                                 mA[1], mB[1], mC[1], mG[0], mU[0], mG[1], mU[1], p));
-    else
-      PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<1> : grouped_gemm_kernel<1>, dim3(grid), dim3(kThreads),
-                                 kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
+    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<1> : grouped_gemm_kernel<1>, dim3(grid), dim3(kThreads),
+                               kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
     count_launch();
   }
 
@@ -1479,12 +1004,8 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; }
     p.nseg = ns;
-    if (mixed)
-      PCOMOE_CUDA_TRY(launch_pdl(grouped_gemm_mixed_kernel<2>, dim3(grid), dim3(kThreads), kSmemDyn, st, mA[0], mB[0], mB[0],
-                                 mA[1], mB[1], mB[1], mB[0], mB[0], mB[1], mB[1], p));
-    else
-      PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<2> : grouped_gemm_kernel<2>, dim3(grid), dim3(kThreads),
-                                 kSmemDyn, st, mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p));
+    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<2> : grouped_gemm_kernel<2>, dim3(grid), dim3(kThreads),
+                               kSmemDyn, st, mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p));
     count_launch();
   }
   PCOMOE_CUDA_TRY(cudaGetLastError());

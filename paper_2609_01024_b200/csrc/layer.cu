@@ -63,7 +63,7 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
   if (n <= 0 || K <= 0 || cfg->hidden <= 0 || cfg->ffn <= 0 || cfg->shared_ffn < 0)
     return PCOMOE_ERR_INVALID_ARG;
   if (cfg->in_dtype != PCOMOE_BF16 && cfg->in_dtype != PCOMOE_FP32) return PCOMOE_ERR_INVALID_ARG;
-  if (cfg->ffn_impl < PCOMOE_FFN_AUTO || cfg->ffn_impl > PCOMOE_FFN_TCGEN05_SWAP)
+  if (cfg->ffn_impl < PCOMOE_FFN_AUTO || cfg->ffn_impl > PCOMOE_FFN_TCGEN05_PAIR)
     return PCOMOE_ERR_INVALID_ARG;
   if (K > n || K > kMaxTopK) return PCOMOE_ERR_SHAPE;
   if (n > kMaxExperts) return PCOMOE_ERR_UNSUPPORTED;
