@@ -125,3 +125,32 @@ def test_large_random_grouping(G, oracle):
         g, st = G.groups_on_gpu(layer, src, tgt, w)
         assert st == 0
         G.assert_groups_equal(g, oracle.groups(src, tgt, w, n, dedup=dedup), T, K)
+
+
+def test_randomised_small_shapes_bit_exact(G, oracle):
+    """Many random (n, K, T, density, lambda) draws, scores quantised to force ties: routing and grouping indices
+    from the GPU equal the oracle's on every one."""
+    rng = np.random.default_rng(2024)
+    for trial in range(40):
+        n = int(rng.integers(2, 10))
+        K = int(rng.integers(1, n + 1))
+        T = int(rng.integers(1, 71))
+        lam = float(rng.choice([0.0, 0.5, 1.0, -0.5]))
+        p = float(rng.uniform(0.1, 1.0))
+        z = rng.standard_normal((T, n)).astype(np.float32)
+        if trial % 2:
+            z = (np.round(z * 2) / 2).astype(np.float32)
+        M = (rng.random((n, n)) < p).astype(np.uint8); np.fill_diagonal(M, 1)
+        Bm = (np.round((-0.5 + 0.5 * rng.standard_normal((n, n))) * 4) / 4).astype(np.float32); np.fill_diagonal(Bm, 0.0)
+        cfg = wl.small_case(trial, T=T, H=64, F=64, n=n, K=K, lam=lam)
+        L = wl.make_layer(cfg, with_weights=False)
+        dedup = trial % 3 != 0
+        layer = G.make_gpu_layer(cfg, L, with_weights=False, mask=M, bias=Bm, lam=lam, dedup=int(dedup))
+        src, tgt, w = G.route_on_gpu(layer, z)
+        rs, rt, rw = oracle.route(z, M, Bm, lam, K)
+        assert np.array_equal(src, rs) and np.array_equal(tgt, rt), (trial, n, K, T)
+        np.testing.assert_allclose(w, rw, rtol=0, atol=1e-6)
+        g, st = G.groups_on_gpu(layer, src, tgt, w)
+        assert st == 0
+        G.assert_groups_equal(g, oracle.groups(src, tgt, w, n, dedup=int(dedup)), T, K)
+        layer.close()
