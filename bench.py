@@ -168,6 +168,8 @@ def main():
                     help="only run warm-up + steps of the device-resident hot path, print a short line and exit")
     ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the hot path from a CUDA graph in the device-resident timing loop")
     ap.add_argument("--ffn-impl", type=int, default=0,
                     help="pcomoe_ffn_impl: 0 auto, 1 SIMT, 2 tcgen05 one CTA per tile, 3 tcgen05 CTA pairs")
     ap.add_argument("--variant", default="default", choices=["default", "vanilla"],
@@ -219,8 +221,14 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps ----
+    step = lambda: layer.forward(d_logits, d_h)
+    if args.graph:
+        step()
+        torch.cuda.synchronize()
+        graph = layer.capture(d_logits, d_h)
+        step = graph.replay
     for _ in range(args.warmup):
-        layer.forward(d_logits, d_h)
+        step()
     assert layer.device_status() == 0, "device reported an error during warm-up"
     if args.profile:
         for _ in range(args.steps):
@@ -238,11 +246,13 @@ def main():
     t_wall0 = time.time()
     e0.record(stream)
     for _ in range(args.steps):
-        layer.forward(d_logits, d_h)
+        step()
     e1.record(stream)
     barrier()
     t_wall1 = time.time()
     launches = B.pcomoe_launch_count() - n0
+    if args.graph:   # replays do not pass through the library's launch counter: count the captured launches
+        m0 = B.pcomoe_launch_count(); layer.forward(d_logits, d_h); launches = (B.pcomoe_launch_count() - m0) * args.steps
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     assert layer.device_status() == 0, "device reported an error during the timed steps"
@@ -313,7 +323,7 @@ def main():
                "vs_baseline": None, "dtype": "bf16" if tc_path else "f32", "data": "synthetic",
                "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
                           "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam,
-                          "R1_over_P": R1 / (cfg.T * cfg.K), "parallelism": f"token-dp{world} (replicas, no collective)",
+                          "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(args.graph), "parallelism": f"token-dp{world} (replicas, no collective)",
                           "l2": "inputs larger than L2 (weights are streamed every step)" if work["weight_bytes"] > 126e6
                                 else "working set fits L2; not a performance target"},
                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},

@@ -303,6 +303,15 @@ class PathMoELayer:
         torch.cuda.current_stream().synchronize()
         return self._pin_y[:T].numpy()
 
+    def capture(self, logits, h, tgt_logits=None):
+        """Records one pass of the hot path on fixed device tensors into a CUDA graph and returns it; every
+        `graph.replay()` then reruns route -> group -> stage 1 -> stage 2 on whatever those tensors hold, with one
+        host call.  Run `forward` once before capturing (first calls set kernel attributes)."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.forward(logits, h, tgt_logits)
+        return g
+
     def stream_from_host(self, pinned_logits, pinned_h, steps: int):
         """Serving loop over `steps` batches that live in PINNED host memory (torch CPU tensors; `pinned_h` is
         bf16 or fp32).  Every step copies its inputs host->device, runs the hot path and copies y device->host;

@@ -137,3 +137,26 @@ def test_streaming_from_pinned_host_buffers(G, oracle):
         y = layer.stream_from_host(pin_logits, pin_h, steps).numpy().copy()
         assert layer.device_status() == 0
         G.check_output(y, yr)
+
+
+def test_cuda_graph_replay_matches_eager(G, oracle):
+    """The whole hot path recorded into a CUDA graph: replays on new inputs give the oracle's outputs."""
+    import torch
+    cfg = wl.small_case(37, T=32, H=256, F=256, n=8, K=2)          # decode-sized: one-CTA kernels, one-block grouping
+    L = wl.make_layer(cfg)
+    layer = G.make_gpu_layer(cfg, L)
+    dl = torch.from_numpy(L.logits).to(layer.device)
+    dh = G.B.to_device(L.h)
+    layer.forward(dl, dh)
+    torch.cuda.synchronize()
+    graph = layer.capture(dl, dh)
+    cfg2 = cfg.scaled(seed=cfg.seed + 1)                            # new tokens, same weights
+    h2 = wl.make_hidden(cfg2); z2 = wl.make_logits(cfg2)
+    dl.copy_(torch.from_numpy(z2)); dh.copy_(G.B.to_device(h2))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    y = layer.y[:cfg.T].cpu().numpy()
+    rs, rt, rw = oracle.route(z2, L.mask, L.bias, cfg.lam, cfg.K)
+    assert np.array_equal(layer.path_src[:cfg.T].cpu().numpy(), rs)
+    G.check_output(y, oracle.ffn(wl.hidden_as_f32(cfg2, h2), L.w_gate, L.w_up, L.w_down, rs, rt, rw))
