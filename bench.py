@@ -49,17 +49,36 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    """Samples SM clocks and throttle reasons (read-only NVML queries, one every few milliseconds from a thread)
+    while the timed region runs; falls back to an nvidia-smi loop when the NVML module is missing."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, uuid=None):
         self.idx = gpu_index
-        self.rows = []
+        self.uuid = uuid
+        self.rows = []          # (time, sm_mhz, max_mhz, set(reasons))
         self.proc = None
+        self.nvml = None
+        self._stop = threading.Event()
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            if self.uuid is not None:
+                u = str(self.uuid)
+                h = pynvml.nvmlDeviceGetHandleByUUID(u if u.startswith("GPU-") else "GPU-" + u)
+            else:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.idx)
+            self.nvml, self.handle = pynvml, h
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                           "-i", str(self.idx), "-lms", "100"], stdout=subprocess.PIPE, text=True)
@@ -68,29 +87,56 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        bits = (("hw_slowdown", n.nvmlClocksEventReasonHwSlowdown if hasattr(n, "nvmlClocksEventReasonHwSlowdown")
+                 else n.nvmlClocksThrottleReasonHwSlowdown),
+                ("hw_thermal_slowdown", getattr(n, "nvmlClocksEventReasonHwThermalSlowdown",
+                                                getattr(n, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40))),
+                ("sw_thermal_slowdown", getattr(n, "nvmlClocksEventReasonSwThermalSlowdown",
+                                                getattr(n, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20))),
+                ("sw_power_cap", getattr(n, "nvmlClocksEventReasonSwPowerCap",
+                                         getattr(n, "nvmlClocksThrottleReasonSwPowerCap", 0x4))))
+        get_reasons = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons",
+                              getattr(n, "nvmlDeviceGetCurrentClocksThrottleReasons", None))
+        while not self._stop.is_set():
+            try:
+                mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                r = int(get_reasons(self.handle)) if get_reasons else 0
+                self.rows.append((time.time(), mhz, self.max_mhz, {name for name, b in bits if r & b}))
+            except Exception:
+                pass
+            time.sleep(0.004)
+
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append((time.time(), line.strip()))
-
-    def stop(self, t0=None, t1=None):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        sm, mx, reasons = [], [], set()
-        for ts, line in self.rows:
-            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
-                continue
-            f = [x.strip() for x in line.split(",")]
+            f = [x.strip() for x in line.strip().split(",")]
             try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
+                rs = {name for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                               "sw_power_cap"), f[4:8]) if v == "Active"}
+                self.rows.append((time.time(), float(f[1]), float(f[2]), rs))
             except Exception:
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
-                if v == "Active":
-                    reasons.add(name)
+
+    def stop(self, t0=None, t1=None):
+        if self.nvml is None and self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["clock sampling unavailable"]}
+        if self.nvml is not None:
+            self._stop.set()
+            self.thread.join(timeout=1.0)
+            pad0, pad1 = 0.0, 0.0
+        else:
+            time.sleep(0.15)
+            self.proc.terminate()
+            pad0, pad1 = 0.05, 0.15
+        sm, mx, reasons = [], [], set()
+        for ts, mhz, mmax, rs in self.rows:
+            if t0 is not None and not (t0 - pad0 <= ts <= t1 + pad1):
+                continue
+            sm.append(mhz); mx.append(mmax); reasons |= rs
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm),
+                "source": "nvml" if self.nvml is not None else "nvidia-smi"}
 
 
 def algorithmic_work(cfg, R1, n_src, n_tgt):
@@ -236,7 +282,11 @@ def main():
         torch.cuda.synchronize()
         print(json.dumps({"profile_run": cfg.name, "steps": args.steps, "status": layer.device_status()}))
         return
-    sampler = ClockSampler(local)
+    try:
+        uuid = torch.cuda.get_device_properties(dev).uuid
+    except Exception:
+        uuid = None
+    sampler = ClockSampler(local, uuid)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)

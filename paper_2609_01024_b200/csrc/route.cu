@@ -224,6 +224,143 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
   }
 }
 
+
+// The same selection with fewer instructions per path, used when the expanded table and a per-warp score
+// cache fit in shared memory.  Table entries are expanded to 16 bytes (byte offsets of z[src] and lambda*u[tgt]
+// inside the warp's row buffer, and the bias), pass 1 keeps every score, pass 2 scans the cached scores four at
+// a time and appends the few that reach the threshold to the candidate list, and the candidates are ranked by
+// counting.  The result is the one the kernel above gives, bit for bit.
+struct FastEntry {
+  uint32_t z_off, u_off;   // byte offsets into the warp's [z | lambda*u] row buffer
+  float bias;
+  uint32_t pad;
+};
+
+template <int KMAX>
+__global__ void __launch_bounds__(256) route_fast_kernel(const RouteParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_grid_wait();
+  const int warps = blockDim.x >> 5;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int A = p.A, A128 = (A + 127) & ~127;
+  float *cache = reinterpret_cast<float *>(smem_raw) + (size_t)warp * A128;          // [warps][A128]
+  FastEntry *st = reinterpret_cast<FastEntry *>(smem_raw + (size_t)warps * A128 * 4);   // [A]
+  float *rows = reinterpret_cast<float *>(st + A) + (size_t)warp * 2 * p.n;            // [warps][2][n]
+  float *cand_s = reinterpret_cast<float *>(st + A) + (size_t)warps * 2 * p.n + warp * 68;   // [warps][68]
+  int *cand_a = reinterpret_cast<int *>(cand_s + 32);
+  int *cand_n = cand_a + 32;
+  for (int a = threadIdx.x; a < A; a += blockDim.x) {
+    const ActiveEntry e = p.table[a];
+    FastEntry f;
+    f.z_off = 4u * e.src;
+    f.u_off = 4u * (p.n + e.tgt);
+    f.bias = e.bias;
+    f.pad = 0;
+    st[a] = f;
+  }
+  for (int a = A + lane; a < A128; a += 32) cache[a] = -INFINITY;   // the tail of the last group of four
+  __syncthreads();
+  const unsigned char *rb = reinterpret_cast<const unsigned char *>(rows);
+  const uint4 *st4 = reinterpret_cast<const uint4 *>(st);
+
+  for (int t = blockIdx.x * warps + warp; t < p.T; t += gridDim.x * warps) {
+    __syncwarp();
+    for (int e = lane; e < p.n; e += 32) {
+      rows[e] = p.z[(size_t)t * p.n + e];
+      rows[p.n + e] = __fmul_rn(p.lambda, p.u[(size_t)t * p.n + e]);
+    }
+    if (lane == 0) *cand_n = 0;
+    __syncwarp();
+
+    // pass 1: every score once, kept in the cache; per-lane maxima
+    float m = -INFINITY;
+#pragma unroll 4
+    for (int a = lane; a < A; a += 32) {
+      const uint4 e = st4[a];
+      const float zi = *reinterpret_cast<const float *>(rb + e.x);
+      const float uj = *reinterpret_cast<const float *>(rb + e.y);
+      const float s = __fadd_rn(__fadd_rn(zi, __uint_as_float(e.z)), uj);
+      cache[a] = s;
+      m = fmaxf(m, s);
+    }
+    // tau = the K-th largest lane maximum: at least K paths score >= tau, so the TopK all do
+    float tau = 0.0f;
+    for (int k = 0; k < p.K; ++k) {
+      tau = warp_max(m);
+      const unsigned hit = __ballot_sync(0xffffffffu, m == tau);
+      if (lane == __ffs(hit) - 1) m = -INFINITY;
+    }
+    __syncwarp();
+    // pass 2: four cached scores per load; the rare ones that reach tau join the candidate list
+    const float4 *c4 = reinterpret_cast<const float4 *>(cache);
+    for (int q = lane; q < (A128 >> 2); q += 32) {
+      const float4 v = c4[q];
+      if (fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)) >= tau) {
+        const float vs[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (vs[c] >= tau && 4 * q + c < A) {
+            const int pos = atomicAdd(cand_n, 1);
+            if (pos < 32) {
+              cand_s[pos] = vs[c];
+              cand_a[pos] = 4 * q + c;
+            }
+          }
+        }
+      }
+    }
+    __syncwarp();
+    const int cnt = *cand_n;
+
+    float my_s = -FLT_MAX;
+    int my_a = 0;
+    if (cnt <= 32) {
+      // rank by counting: the position of a candidate is the number of candidates that rank before it
+      const float cs = lane < cnt ? cand_s[lane] : -INFINITY;
+      const int ca = lane < cnt ? cand_a[lane] : 0x7fffffff;
+      int rank = 0;
+      for (int j = 0; j < cnt; ++j) {
+        const float os = __shfl_sync(0xffffffffu, cs, j);
+        const int oa = __shfl_sync(0xffffffffu, ca, j);
+        rank += ranks_before(os, oa, cs, ca) ? 1 : 0;
+      }
+      __syncwarp();
+      if (lane < cnt && rank < p.K) {   // rank order onto lanes 0..K-1, through the candidate buffer
+        cand_s[rank] = cs;
+        cand_a[rank] = ca;
+      }
+      __syncwarp();
+      if (lane < p.K) {
+        my_s = cand_s[lane];
+        my_a = cand_a[lane];
+      }
+    } else {
+      RouteParams q = p;      // the row buffer already holds lambda*u: the lists multiply by one
+      q.lambda = 1.0f;
+      topk_by_lists<KMAX>(q, p.table, rows, rows + p.n, lane, my_s, my_a);
+    }
+
+    const float s0 = __shfl_sync(0xffffffffu, my_s, 0);
+    float e = lane < p.K ? expf(my_s - s0) : 0.0f;
+    float den;
+    if (p.norm_topk) {
+      den = e;
+    } else {
+      den = 0.0f;
+      for (int a = lane; a < A; a += 32) den += expf(cache[a] - s0);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
+    if (lane < p.K) {
+      const ActiveEntry en = p.table[my_a];
+      const size_t o = (size_t)t * p.K + lane;
+      p.src[o] = en.src;
+      p.tgt[o] = en.tgt;
+      p.w[o] = e / den * p.scale;
+    }
+  }
+}
+
 pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, const float *u,
                            int32_t *src, int32_t *tgt, float *w, cudaStream_t st) {
   const pcomoe_config &c = L->cfg;
@@ -233,23 +370,41 @@ pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, con
   p.T = T; p.n = c.n_experts; p.K = c.top_k; p.A = L->n_active;
   p.lambda = c.lambda; p.scale = c.routed_scale; p.norm_topk = c.norm_topk;
   const int threads = 256, warps = threads / 32;
-  size_t smem = ((size_t)warps * (2 * p.n + 64) * 4 + 15) & ~size_t(15);
-  const size_t tab_bytes = sizeof(ActiveEntry) * (size_t)p.A;
-  p.table_in_smem = smem + tab_bytes <= 160 * 1024;
-  if (p.table_in_smem) smem += (tab_bytes + 15) & ~size_t(15);
-  const size_t cache_bytes = (size_t)warps * ((p.A + 31) / 32 * 32) * 4;
-  p.cache_scores = smem + cache_bytes <= 100 * 1024;
-  if (p.cache_scores) smem += cache_bytes;
-  int grid = (T + warps - 1) / warps;
-  const int cap = L->sm_count * 4;
-  if (grid > cap) grid = cap;
-
+  const int cap_rows = (T + warps - 1) / warps;
+  // fast kernel: expanded table + per-warp score cache + row and candidate buffers in shared memory
+  const size_t a128 = ((size_t)p.A + 127) & ~size_t(127);
+  const size_t smem_fast = (size_t)warps * a128 * 4 + (size_t)p.A * sizeof(FastEntry) +
+                           (size_t)warps * (2 * p.n + 68) * 4;
   void (*kern)(const RouteParams) = nullptr;
-  if (p.K <= 2) kern = route_kernel<2>;
-  else if (p.K <= 4) kern = route_kernel<4>;
-  else if (p.K <= 8) kern = route_kernel<8>;
-  else if (p.K <= 16) kern = route_kernel<16>;
-  else kern = route_kernel<32>;
+  size_t smem;
+  if (smem_fast <= 100 * 1024) {
+    smem = smem_fast;
+    p.table_in_smem = 1;
+    p.cache_scores = 1;
+    if (p.K <= 2) kern = route_fast_kernel<2>;
+    else if (p.K <= 4) kern = route_fast_kernel<4>;
+    else if (p.K <= 8) kern = route_fast_kernel<8>;
+    else if (p.K <= 16) kern = route_fast_kernel<16>;
+    else kern = route_fast_kernel<32>;
+  } else {
+    smem = ((size_t)warps * (2 * p.n + 64) * 4 + 15) & ~size_t(15);
+    const size_t tab_bytes = sizeof(ActiveEntry) * (size_t)p.A;
+    p.table_in_smem = smem + tab_bytes <= 160 * 1024;
+    if (p.table_in_smem) smem += (tab_bytes + 15) & ~size_t(15);
+    const size_t cache_bytes = (size_t)warps * ((p.A + 31) / 32 * 32) * 4;
+    p.cache_scores = smem + cache_bytes <= 100 * 1024;
+    if (p.cache_scores) smem += cache_bytes;
+    if (p.K <= 2) kern = route_kernel<2>;
+    else if (p.K <= 4) kern = route_kernel<4>;
+    else if (p.K <= 8) kern = route_kernel<8>;
+    else if (p.K <= 16) kern = route_kernel<16>;
+    else kern = route_kernel<32>;
+  }
+  // as many blocks as stay resident together (the token loop strides over the grid)
+  int per_sm = (int)((227 * 1024) / (smem + 1024));
+  per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+  int grid = cap_rows;
+  if (grid > L->sm_count * per_sm) grid = L->sm_count * per_sm;
   if (smem > 48 * 1024)
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   PCOMOE_CUDA_TRY(launch_pdl(kern, dim3(grid), dim3(threads), smem, st, p));
