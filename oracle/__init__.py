@@ -170,3 +170,28 @@ def ffn_grouped(h, w_gate, w_up, w_down, g):
     if rc != 0:
         raise ValueError(f"pcomoe_oracle_ffn_grouped failed with code {rc}")
     return y
+
+
+def router_logits(h, w_router, lora_a=None, lora_b=None, lora_scale=1.0):
+    """logits [T,n] in fp64: h W_r^T (+ scale * (h A^T) B^T).  ``h`` fp32 [T,H]; ``w_router`` [n,H] and ``lora_a``
+    [r,H] fp32 or bf16 bit patterns (one type); ``lora_b`` [n,r] fp32."""
+    h = _c(h, np.float32)
+    T, H = h.shape
+    w = np.ascontiguousarray(w_router)
+    n = w.shape[0]
+    wd = _wdtype(w)
+    if lora_a is not None:
+        a = np.ascontiguousarray(lora_a)
+        assert _wdtype(a) == wd and a.shape[1] == H
+        b = _c(lora_b, np.float32)
+        r = a.shape[0]
+        assert b.shape == (n, r)
+    else:
+        a, b, r = None, None, 0
+    out = np.zeros((T, n), np.float64)
+    rc = _load().pcomoe_oracle_router_logits(ctypes.c_int32(T), ctypes.c_int32(H), ctypes.c_int32(n),
+                                             ctypes.c_int32(r), _p(h), _p(w), _p(a), _p(b),
+                                             ctypes.c_double(lora_scale), ctypes.c_int32(wd), _p(out))
+    if rc != 0:
+        raise ValueError(f"pcomoe_oracle_router_logits failed with code {rc}")
+    return out

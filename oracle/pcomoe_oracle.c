@@ -351,3 +351,35 @@ int pcomoe_oracle_mask_from_bias(int32_t n, const float *B, int64_t keep, uint8_
   }
   return ORACLE_OK;
 }
+
+/* ---------------------------------------------------------------------------
+ * Router in front of the path gate (Sec. 3.1: the router turns the hidden state into routing scores;
+ * Sec. 4.2 names them the base routing signal g_base(h), and g_tgt(h) when a second head is given):
+ *   logits[t,e] = sum_k h[t,k] * W_r[e,k]
+ * plus, when a low-rank gate adaptation is attached (Sec. 5.1: rank-16 LoRA on the gate),
+ *   logits[t,e] += scale * sum_q B_l[e,q] * (sum_k A_l[q,k] * h[t,k]).
+ * h [T,H] fp32; W_r [n,H] and A_l [r,H] in wdtype; B_l [n,r] fp32; logits [T,n] fp64.  r = 0: no adaptation.
+ * The paper gives no precision for the router: everything here is fp64 from the stored values.
+ * ------------------------------------------------------------------------- */
+int pcomoe_oracle_router_logits(int32_t T, int32_t H, int32_t n, int32_t r, const float *h, const void *Wr,
+                                const void *Al, const float *Bl, double scale, int32_t wdtype,
+                                double *logits) {
+  if (T < 0 || H <= 0 || n <= 0 || r < 0 || !h || !Wr || !logits) return ORACLE_ERR_ARG;
+  if (r > 0 && (!Al || !Bl)) return ORACLE_ERR_ARG;
+  if (wdtype != ORACLE_W_F32 && wdtype != ORACLE_W_BF16) return ORACLE_ERR_ARG;
+#pragma omp parallel for schedule(static)
+  for (int32_t t = 0; t < T; ++t) {
+    double *x = (double *)malloc(sizeof(double) * (size_t)(H + (r > 0 ? r : 1)));
+    double *low = x + H;
+    for (int32_t k = 0; k < H; ++k) x[k] = (double)h[(size_t)t * H + k];
+    for (int32_t q = 0; q < r; ++q) low[q] = dot_row(Al, (size_t)q * H, x, H, wdtype);
+    for (int32_t e = 0; e < n; ++e) {
+      double v = dot_row(Wr, (size_t)e * H, x, H, wdtype);
+      double d = 0.0;
+      for (int32_t q = 0; q < r; ++q) d += (double)Bl[(size_t)e * r + q] * low[q];
+      logits[(size_t)t * n + e] = v + scale * d;
+    }
+    free(x);
+  }
+  return ORACLE_OK;
+}

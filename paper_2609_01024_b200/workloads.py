@@ -25,6 +25,7 @@ import numpy as np
 # gate, up, down, shared)
 T_MASK, T_BIAS, T_ROUTER, T_LOGITS, T_HIDDEN, T_GATE, T_UP, T_DOWN = range(8)
 T_SH_GATE, T_SH_UP, T_SH_DOWN, T_PERM, T_TGT_LOGITS = range(8, 13)
+T_ROUTER_W, T_LORA_A, T_LORA_B = range(13, 16)
 
 
 @dataclasses.dataclass(frozen=True)
@@ -142,6 +143,22 @@ def make_tgt_logits(cfg: LayerConfig) -> np.ndarray:
     """A separate projection-side prior g_tgt [T,n] (used only by tests of the
     optional second-gate input)."""
     return _normal(cfg.seed, T_TGT_LOGITS, 0, (cfg.T, cfg.n), cfg.sigma_z)
+
+
+def make_router_weights(cfg: LayerConfig, lora_rank: int = 0):
+    """Router in front of the path gate: W_r [n,H] in the layer's storage type, scaled so that the logits of
+    unit-variance hidden states have standard deviation sigma_z; with ``lora_rank`` r > 0 also a low-rank
+    gate adaptation A [r,H] (storage type) and B [n,r] (fp32) whose delta is about a quarter of that size.
+    Returns (W_r, A, B); A and B are None when r == 0."""
+    s = cfg.sigma_z / (cfg.hidden_std * np.sqrt(cfg.H))
+    w = _normal(cfg.seed, T_ROUTER_W, 0, (cfg.n, cfg.H), s)
+    w = w if cfg.dtype == "f32" else f32_to_bf16_bits(w)
+    if lora_rank <= 0:
+        return w, None, None
+    a = _normal(cfg.seed, T_LORA_A, 0, (lora_rank, cfg.H), 1.0 / (cfg.hidden_std * np.sqrt(cfg.H)))
+    a = a if cfg.dtype == "f32" else f32_to_bf16_bits(a)
+    b = _normal(cfg.seed, T_LORA_B, 0, (cfg.n, lora_rank), 0.25 * cfg.sigma_z / np.sqrt(lora_rank))
+    return w, a, np.ascontiguousarray(b, dtype=np.float32)
 
 
 def _std(cfg: LayerConfig, fan_in: int) -> float:
