@@ -214,6 +214,9 @@ def main():
                     help="only run warm-up + steps of the device-resident hot path, print a short line and exit")
     ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--router", type=int, default=-1,
+                    help="r >= 0: the timed step starts from hidden states (router GEMM with a rank-r gate adaptation, "
+                         "0 = none, in front of the path gate); default -1: logits are an input, as the metric is quoted")
     ap.add_argument("--graph", action="store_true",
                     help="replay the hot path from a CUDA graph in the device-resident timing loop")
     ap.add_argument("--ffn-impl", type=int, default=0,
@@ -268,6 +271,12 @@ def main():
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps ----
     step = lambda: layer.forward(d_logits, d_h)
+    if args.router >= 0:
+        w_r, l_a, l_b = wl.make_router_weights(cfg, lora_rank=args.router)
+        layer.set_router(B.to_device(w_r, dev), B.to_device(l_a, dev),
+                         None if l_b is None else torch.from_numpy(l_b).to(dev), 1.0)
+        step = lambda: layer.forward_hidden(d_h)
+        assert not args.graph, "--graph records the logits-in path"
     if args.graph:
         step()
         torch.cuda.synchronize()
@@ -330,10 +339,12 @@ def main():
     n_src = cfg.n - int(stats[4]); n_tgt = cfg.n - int(stats[5])
     work = algorithmic_work(cfg, R1, n_src, n_tgt)
     stage_ms = {}
-    for name, fn in (("route", lambda: layer.route(d_logits)), ("groups", lambda: layer.build_groups(cfg.T)),
+    for name, fn in (("router", lambda: layer.router_logits(d_h)), ("route", lambda: layer.route(d_logits)), ("groups", lambda: layer.build_groups(cfg.T)),
                      ("stage1_routed", lambda: layer.ffn_stages(d_h, 1)), ("stage1_shared", lambda: layer.ffn_stages(d_h, 2)),
                      ("stage2_routed", lambda: layer.ffn_stages(d_h, 4)), ("stage2_shared", lambda: layer.ffn_stages(d_h, 8))):
         if "shared" in name and not cfg.F_sh:
+            continue
+        if name == "router" and args.router < 0:
             continue
         ts = []
         for i in range(3 + args.steps):
@@ -373,7 +384,10 @@ def main():
                "vs_baseline": None, "dtype": "bf16" if tc_path else "f32", "data": "synthetic",
                "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
                           "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam,
-                          "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(args.graph), "parallelism": f"token-dp{world} (replicas, no collective)",
+                          "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(args.graph),
+                          "router_in_step": (f"yes (rank-{args.router} gate adaptation)" if args.router > 0 else
+                                             "yes" if args.router == 0 else "no (logits are an input)"),
+                          "parallelism": f"token-dp{world} (replicas, no collective)",
                           "l2": "inputs larger than L2 (weights are streamed every step)" if work["weight_bytes"] > 126e6
                                 else "working set fits L2; not a performance target"},
                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},

@@ -102,6 +102,18 @@ pcomoe_status pcomoe_layer_destroy(pcomoe_layer *layer);
  */
 pcomoe_status pcomoe_mask_from_bias(int32_t n, const float *h_bias, float keep_fraction, uint8_t *h_mask);
 
+/*
+ * Host utility: one step of the progressive tightening of a layer's mask (Sec. 4.2: the sparsity criterion is
+ * tightened at training intervals, the active path set only contracts, m_ii = 1 is hard-coded).  Of the
+ * off-diagonal pairs active in h_prev_mask, the share keep_fraction (nearest count) with the largest current
+ * bias stays active, ties to the smaller flat id; pairs dropped earlier never return, whatever their bias has
+ * become.  h_mask [n*n] may be the same array as h_prev_mask.  The paper states neither the criterion nor the
+ * schedule: a schedule is a sequence of calls, one per interval, each with that interval's bias.
+ * Errors: INVALID_ARG (NULL, n <= 0, keep_fraction outside [0,1] or not finite).
+ */
+pcomoe_status pcomoe_mask_tighten(int32_t n, const float *h_bias, const uint8_t *h_prev_mask, float keep_fraction,
+                                  uint8_t *h_mask);
+
 /* Number of active paths |A| of the layer; copies up to `cap` table entries to host arrays
  * (any of them may be NULL).  For checking the table against the mask. */
 pcomoe_status pcomoe_layer_active_set(const pcomoe_layer *layer, int32_t cap, int32_t *h_src,
@@ -227,8 +239,30 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, co
                                         const pcomoe_groups *groups, void *d_y, void *d_workspace,
                                         size_t ws_bytes, void *stream, int32_t stages);
 
-/* Synchronises `stream`, reads the workspace's status word and returns the first error a kernel
- * recorded (PCOMOE_OK if none); the word is cleared by the next pcomoe_build_path_groups. */
+/* Router in front of the path gate (Sec. 3.1: the router maps a token's hidden state to routing scores;
+ * Sec. 4.2 uses them as the base routing signal g_base(h), and as g_tgt(h) unless a second head is given):
+ *     d_logits[t,e] = sum_k d_h[t,k] * d_w_router[e,k]
+ * and, with a rank-r gate adaptation attached (Sec. 5.1 fine-tunes the gate with rank-16 LoRA),
+ *     d_logits[t,e] += lora_scale * sum_q d_lora_b[e,q] * (sum_k d_lora_a[q,k] * d_h[t,k]).
+ * The output feeds pcomoe_route_paths (call it again with a second weight for a separate target head).
+ *   d_h        [T,H]  in_dtype, device          d_w_router [n,H]  in_dtype, device
+ *   d_lora_a   [r,H]  in_dtype, device or NULL  d_lora_b   [n,r]  fp32, device or NULL   (both when r > 0)
+ *   d_logits   [T,n]  fp32, device, written     lora_rank  r >= 0 (0: no adaptation)
+ * Products are exact in fp32 (bf16 inputs) and summed in fp32; one thread block owns a tile of 128 tokens from
+ * start to end, so the logits are the same bits on every call.  bf16 layers with H % 8 == 0, H >= 64 and
+ * (n rounded up to 8) + r <= 256, r <= 64 run on the tensor cores; everything else takes a plain kernel.
+ * Asynchronous on `stream`; allocates nothing.  The workspace only receives the router's device status word
+ * (a wait that ran out -> TIMEOUT), which this call clears first and pcomoe_device_status reports.
+ * Errors: INVALID_ARG (NULL pointers, r < 0), SHAPE (T < 0, r > 256), WORKSPACE, UNSUPPORTED (plain kernel:
+ * H too large for shared memory), CUDA. */
+pcomoe_status pcomoe_router_logits(const pcomoe_layer *layer, int32_t T, const void *d_h,
+                                   const void *d_w_router, const void *d_lora_a, const float *d_lora_b,
+                                   int32_t lora_rank, float lora_scale, float *d_logits, void *d_workspace,
+                                   size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, reads the workspace's status words and returns the first error a kernel
+ * recorded (PCOMOE_OK if none): the layer's word is cleared by the next pcomoe_build_path_groups, the
+ * router's by the next pcomoe_router_logits. */
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream);
 
 /* Launch counters (kernels and memsets enqueued by this library since load, per process). */

@@ -71,6 +71,17 @@ def mask_from_bias(bias, keep: int):
     return m
 
 
+def mask_tighten(bias, prev_mask, keep: int):
+    b = _c(bias, np.float32)
+    pm = _c(prev_mask, np.uint8)
+    n = b.shape[0]
+    m = np.zeros((n, n), np.uint8)
+    rc = _load().pcomoe_oracle_mask_tighten(ctypes.c_int32(n), _p(b), _p(pm), ctypes.c_int64(keep), _p(m))
+    if rc != 0:
+        raise ValueError(f"pcomoe_oracle_mask_tighten failed with code {rc}")
+    return m
+
+
 def route(logits, mask, bias, lam, K, tgt_logits=None, norm_topk=1, routed_scale=1.0, with_scores=False):
     z = _c(logits, np.float32)
     u = z if tgt_logits is None else _c(tgt_logits, np.float32)

@@ -383,3 +383,28 @@ int pcomoe_oracle_router_logits(int32_t T, int32_t H, int32_t n, int32_t r, cons
   }
   return ORACLE_OK;
 }
+
+/* ---------------------------------------------------------------------------
+ * One step of the progressive tightening (Sec. 4.2: the sparsity criterion is tightened at training intervals
+ * and the active path set only contracts; the diagonal always stays).  Reading: of the off-diagonal pairs
+ * active in M_prev, the `keep` with the largest current bias stay active (ties to the smaller flat id); a pair
+ * that was dropped earlier never returns.  Repeated arg-max, plain and slow.
+ * ------------------------------------------------------------------------- */
+int pcomoe_oracle_mask_tighten(int32_t n, const float *B, const uint8_t *M_prev, int64_t keep, uint8_t *M) {
+  if (n <= 0 || keep < 0) return ORACLE_ERR_ARG;
+  int64_t active = 0;
+  for (int32_t p = 0; p < n * n; ++p)
+    if (p / n != p % n && M_prev[p]) ++active;
+  if (keep > active) return ORACLE_ERR_ARG;
+  for (int32_t p = 0; p < n * n; ++p) M[p] = 0;
+  for (int32_t i = 0; i < n; ++i) M[(size_t)i * n + i] = 1;
+  for (int64_t r = 0; r < keep; ++r) {
+    int32_t best = -1;
+    for (int32_t p = 0; p < n * n; ++p) {
+      if (p / n == p % n || !M_prev[p] || M[p]) continue;
+      if (best < 0 || B[p] > B[best]) best = p;
+    }
+    M[best] = 1;
+  }
+  return ORACLE_OK;
+}

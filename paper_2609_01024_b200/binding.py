@@ -20,9 +20,9 @@ STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_WORKSPACE
 PCOMOE_BF16, PCOMOE_FP32 = 0, 1
 PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR = 0, 1, 2, 3
 
-EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
+EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_mask_tighten", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
            "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",
-           "pcomoe_ffn_forward_stages",
+           "pcomoe_ffn_forward_stages", "pcomoe_router_logits",
            "pcomoe_device_status",
            "pcomoe_launch_count", "pcomoe_status_string"]
 
@@ -61,6 +61,7 @@ def load_library(path: str | None = None):
     vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
     lib.pcomoe_layer_create.argtypes = [ctypes.POINTER(pcomoe_config), vp, vp, ctypes.POINTER(vp)]
     lib.pcomoe_mask_from_bias.argtypes = [i32, vp, ctypes.c_float, vp]
+    lib.pcomoe_mask_tighten.argtypes = [i32, vp, vp, ctypes.c_float, vp]
     lib.pcomoe_layer_destroy.argtypes = [vp]
     lib.pcomoe_layer_active_set.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(i32)]
     lib.pcomoe_workspace_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
@@ -69,6 +70,7 @@ def load_library(path: str | None = None):
     lib.pcomoe_build_path_groups_static.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp]
     lib.pcomoe_ffn_forward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
     lib.pcomoe_ffn_forward_stages.argtypes = lib.pcomoe_ffn_forward.argtypes + [i32]
+    lib.pcomoe_router_logits.argtypes = [vp, i32, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, sz, vp]
     lib.pcomoe_device_status.argtypes = [vp, vp]
     lib.pcomoe_launch_count.restype = ctypes.c_int64
     lib.pcomoe_status_string.restype = ctypes.c_char_p
@@ -117,6 +119,19 @@ def pcomoe_mask_from_bias(bias, keep_fraction: float) -> np.ndarray:
     m = np.zeros((n, n), np.uint8)
     _check(load_library().pcomoe_mask_from_bias(n, b.ctypes.data_as(ctypes.c_void_p), ctypes.c_float(keep_fraction),
                                                 m.ctypes.data_as(ctypes.c_void_p)), "pcomoe_mask_from_bias")
+    return m
+
+
+def pcomoe_mask_tighten(bias, prev_mask, keep_fraction: float) -> np.ndarray:
+    """Host utility: one tightening step - of the off-diagonal paths active in `prev_mask`, the `keep_fraction`
+    with the largest bias stay active."""
+    b = np.ascontiguousarray(bias, dtype=np.float32)
+    pm = np.ascontiguousarray(prev_mask, dtype=np.uint8)
+    n = b.shape[0]
+    m = np.zeros((n, n), np.uint8)
+    _check(load_library().pcomoe_mask_tighten(n, b.ctypes.data_as(ctypes.c_void_p), pm.ctypes.data_as(ctypes.c_void_p),
+                                              ctypes.c_float(keep_fraction), m.ctypes.data_as(ctypes.c_void_p)),
+           "pcomoe_mask_tighten")
     return m
 
 
@@ -207,6 +222,13 @@ def pcomoe_ffn_forward_stages(layer, T, h, w_gate, w_up, w_down, wsh_gate, wsh_u
                                                     stages), "pcomoe_ffn_forward_stages")
 
 
+def pcomoe_router_logits(layer, T, h, w_router, lora_a, lora_b, lora_rank: int, lora_scale: float, logits, workspace):
+    _check(load_library().pcomoe_router_logits(layer, T, _ptr(h), _ptr(w_router), _ptr(lora_a), _ptr(lora_b),
+                                               lora_rank, lora_scale, _ptr(logits), _ptr(workspace),
+                                               workspace.numel() * workspace.element_size(), _stream()),
+           "pcomoe_router_logits")
+
+
 def pcomoe_device_status(workspace) -> int:
     return int(load_library().pcomoe_device_status(_ptr(workspace), _stream()))
 
@@ -269,6 +291,24 @@ class PathMoELayer:
         T = h.shape[0]
         pcomoe_ffn_forward_stages(self.layer, T, h, self.w_gate, self.w_up, self.w_down, *self.shared, self.groups,
                                   self.y, self.workspace, stages)
+
+    def set_router(self, w_router, lora_a=None, lora_b=None, lora_scale: float = 1.0):
+        """Attaches a router (device tensors: w_router [n,H] and lora_a [r,H] in the layer's type, lora_b [n,r]
+        fp32) so that `router_logits` / `forward_hidden` can start from hidden states."""
+        self.w_router, self.lora_a, self.lora_b, self.lora_scale = w_router, lora_a, lora_b, float(lora_scale)
+        self.lora_rank = 0 if lora_a is None else int(lora_a.shape[0])
+        self.logits = torch.empty(self.max_tokens, self.n, dtype=torch.float32, device=self.device)
+
+    def router_logits(self, h):
+        T = h.shape[0]
+        assert T <= self.max_tokens
+        pcomoe_router_logits(self.layer, T, h, self.w_router, self.lora_a, self.lora_b, self.lora_rank,
+                             self.lora_scale, self.logits, self.workspace)
+        return self.logits[:T]
+
+    def forward_hidden(self, h):
+        """Router -> route -> group -> stage 1 -> stage 2, from hidden states alone."""
+        return self.forward(self.router_logits(h), h)
 
     def forward(self, logits, h, tgt_logits=None):
         """The whole hot path on device tensors: route -> group -> stage 1 -> stage 2.  Returns y [T,H] fp32."""

@@ -30,7 +30,9 @@ struct DevPlan {
   int32_t empty1;      // sources without rows
   int32_t empty2;      // targets without rows
   int32_t T;           // tokens of the last pcomoe_build_path_groups
+  int32_t status_router;   // first error of the router kernel; not cleared by the grouping step
 };
+constexpr size_t kPlanClearBytes = 32;   // what the grouping step zeroes: everything before status_router
 
 // Byte offsets of the workspace sections (all multiples of 256).
 struct WsLayout {
@@ -117,6 +119,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // launchers implemented in the kernel translation units
 pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, const float *u,
                            int32_t *src, int32_t *tgt, float *w, cudaStream_t st);
+pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, const void *w_router,
+                            const void *lora_a, const float *lora_b, int32_t r, float scale, float *logits,
+                            int32_t *status, cudaStream_t st);
 pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src, const int32_t *tgt,
                             const float *w, const pcomoe_groups *g, char *ws, const WsLayout &lay,
                             cudaStream_t st);

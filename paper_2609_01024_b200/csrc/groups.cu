@@ -311,7 +311,7 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
     return PCOMOE_OK;
   }
   // the status word and the plan start from zero
-  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.plan, 0, sizeof(DevPlan), st));
+  PCOMOE_CUDA_TRY(cudaMemsetAsync(ws + lay.plan, 0, kPlanClearBytes, st));
   PCOMOE_CUDA_TRY(launch_pdl(group_count_kernel, dim3(p.nb), dim3(p.chunk), smem_count, st, p));
   count_launch(2);
   PCOMOE_CUDA_TRY(launch_pdl(group_colscan_kernel, dim3((2 * p.n + 3) / 4), dim3(128), 0, st, p));

@@ -140,6 +140,23 @@ pcomoe_status pcomoe_mask_from_bias(int32_t n, const float *h_bias, float keep_f
   return PCOMOE_OK;
 }
 
+pcomoe_status pcomoe_mask_tighten(int32_t n, const float *h_bias, const uint8_t *h_prev_mask, float keep_fraction,
+                                  uint8_t *h_mask) {
+  if (n <= 0 || !h_bias || !h_prev_mask || !h_mask || !(keep_fraction >= 0.0f && keep_fraction <= 1.0f))
+    return PCOMOE_ERR_INVALID_ARG;
+  std::vector<int32_t> order;
+  for (int32_t i = 0; i < n; ++i)
+    for (int32_t j = 0; j < n; ++j)
+      if (i != j && h_prev_mask[(size_t)i * n + j]) order.push_back(i * n + j);
+  const int64_t keep = (int64_t)std::llround((double)keep_fraction * (double)order.size());
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return h_bias[a] > h_bias[b]; });
+  std::vector<uint8_t> m((size_t)n * n, 0);          // built aside: h_mask may be h_prev_mask
+  for (int32_t i = 0; i < n; ++i) m[(size_t)i * n + i] = 1;
+  for (int64_t r = 0; r < keep; ++r) m[(size_t)order[(size_t)r]] = 1;
+  std::memcpy(h_mask, m.data(), m.size());
+  return PCOMOE_OK;
+}
+
 pcomoe_status pcomoe_layer_destroy(pcomoe_layer *L) {
   if (!L) return PCOMOE_ERR_INVALID_ARG;
   if (L->d_table) cudaFree(L->d_table);
@@ -239,12 +256,31 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *L, int32_t T, const 
                          groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
 }
 
+pcomoe_status pcomoe_router_logits(const pcomoe_layer *L, int32_t T, const void *d_h, const void *d_w_router,
+                                   const void *d_lora_a, const float *d_lora_b, int32_t lora_rank,
+                                   float lora_scale, float *d_logits, void *d_workspace, size_t ws_bytes,
+                                   void *stream) {
+  if (!L || lora_rank < 0) return PCOMOE_ERR_INVALID_ARG;
+  if (T < 0) return PCOMOE_ERR_SHAPE;
+  if (T == 0) return PCOMOE_OK;
+  if (!d_h || !d_w_router || !d_logits) return PCOMOE_ERR_INVALID_ARG;
+  if (lora_rank > 0 && (!d_lora_a || !d_lora_b)) return PCOMOE_ERR_INVALID_ARG;
+  if (lora_rank > 256) return PCOMOE_ERR_SHAPE;
+  WsLayout lay;
+  pcomoe_status s = check_ws(L, T, d_workspace, ws_bytes, &lay);
+  if (s != PCOMOE_OK) return s;
+  DevPlan *plan = reinterpret_cast<DevPlan *>((char *)d_workspace + lay.plan);
+  return launch_router(L, T, d_h, d_w_router, d_lora_a, d_lora_b, lora_rank, lora_scale, d_logits,
+                       &plan->status_router, (cudaStream_t)stream);
+}
+
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream) {
   if (!d_workspace) return PCOMOE_ERR_WORKSPACE;
-  int32_t st = 0;
+  DevPlan plan;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return PCOMOE_ERR_CUDA;
-  if (cudaMemcpy(&st, d_workspace, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+  if (cudaMemcpy(&plan, d_workspace, sizeof(DevPlan), cudaMemcpyDeviceToHost) != cudaSuccess)
     return PCOMOE_ERR_CUDA;
+  const int32_t st = plan.status ? plan.status : plan.status_router;
   if (st < 0 || st > PCOMOE_ERR_INDEX) return PCOMOE_ERR_CUDA;
   return (pcomoe_status)st;
 }

@@ -1,0 +1,275 @@
+// K0: the router in front of the path gate (Sec. 3.1: the router turns a token's hidden state into routing
+// scores; Sec. 4.2 calls them the base routing signal g_base(h)):
+//     logits[t,e] = sum_k h[t,k] W_r[e,k]   (+ scale * sum_q B_l[e,q] * sum_k A_l[q,k] h[t,k], the rank-r gate
+//                                              adaptation of Sec. 5.1)
+// The work is a skinny GEMM bound by one read of h, so a tile is 128 tokens x all experts: one CTA streams its
+// 128 rows of h through a 4-stage TMA ring while W_r (and A_l, stacked under it as extra output columns) comes
+// from L2, one thread issues tcgen05.mma (M 128, N = padded n + r, bf16 in, fp32 accumulate in TMEM), and the
+// epilogue turns the accumulators around through shared memory, applies the low-rank term and writes fp32
+// logits coalesced.  One CTA owns a tile from start to end (no split-K, no atomics): logits are reproducible
+// bit for bit, which matters because they decide the TopK.
+// Layers that are not bf16 (or whose shapes the tile does not cover) take a plain SIMT kernel.
+#include <cuda_bf16.h>
+
+#include "tc_ptx.cuh"
+
+namespace pcomoe {
+namespace {
+
+constexpr int kRStages = 4;
+constexpr uint32_t kRA = kTileM * BK * 2;            // 16 KB of h per k-block
+constexpr uint32_t kRB = 256 * BK * 2;               // up to 256 stacked weight rows per k-block
+constexpr uint32_t kRStage = kRA + kRB;
+constexpr size_t kRSmem = (size_t)kRStages * kRStage + 1024;
+constexpr int kRThreads = 192;
+
+struct RouterParams {
+  float *logits;          // [T,n]
+  const float *lora_b;    // [n,r] or NULL
+  int32_t *status;        // device status word of the router (may be NULL)
+  int32_t T, n, r, n8;    // n8: row of the stacked tile where A_l starts (n rounded up to 8)
+  int32_t n_mma;          // MMA N: n8 + r rounded up to 16
+  int32_t kb;             // k-blocks
+  uint32_t idesc, tmem_cols;
+  float scale;
+};
+
+__device__ __forceinline__ void umma_bf16_n(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kRThreads, 1)
+router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
+                   const __grid_constant__ CUtensorMap tmL, const RouterParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  pdl_grid_wait();
+  __shared__ __align__(8) uint64_t s_bar[2 * kRStages + 1];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ float s_lb[64 * 64];                      // B_l when it fits (n*r <= 4096), else read from global
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char *ring_ptr = smem_dyn + (ring - smem_u32(smem_dyn));
+  const uint32_t bar0 = smem_u32(s_bar);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kRStages + s); };
+  const uint32_t acc_bar = bar0 + 8u * (2 * kRStages);
+  const bool lb_smem = p.r > 0 && p.n * p.r <= 64 * 64;
+
+  // rows of the stacked weight tile that no load writes (padding up to the MMA's N) start as zeros
+  for (int s = 0; s < kRStages; ++s) {
+    uint4 *b = reinterpret_cast<uint4 *>(ring_ptr + (size_t)s * kRStage + kRA);
+    for (int i = threadIdx.x; i < p.n_mma * 8; i += blockDim.x) b[i] = make_uint4(0, 0, 0, 0);
+  }
+  if (lb_smem)
+    for (int i = threadIdx.x; i < p.n * p.r; i += blockDim.x) s_lb[i] = p.lora_b[i];
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < kRStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(acc_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem;
+  volatile int *abort_flag = &s_abort;
+  const int row0 = blockIdx.x * kTileM;
+  const uint32_t stage_tx = kRA + (uint32_t)(p.n + p.r) * (BK * 2);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int kb = 0; kb < p.kb; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
+        const uint32_t sa = ring + stage * kRStage, sb = sa + kRA;
+        mbar_arrive_expect_tx(full_bar(stage), stage_tx);
+        tma_load_2d(sa, &tmH, kb * BK, row0, full_bar(stage));
+        tma_load_2d(sb, &tmW, kb * BK, 0, full_bar(stage));
+        if (p.r > 0) tma_load_2d(sb + (uint32_t)p.n8 * (BK * 2), &tmL, kb * BK, 0, full_bar(stage));
+        if (++stage == kRStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int kb = 0; kb < p.kb; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t sa = ring + stage * kRStage, sb = sa + kRA;
+        const uint64_t da = umma_desc(sa), db = umma_desc(sb);
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k)
+          umma_bf16_n(tmem_base, da + 2u * k, db + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+        umma_commit(empty_bar(stage));
+        if (++stage == kRStages) { stage = 0; phase ^= 1u; }
+      }
+      if (alive) umma_commit(acc_bar);
+    }
+    __syncwarp();
+  }
+  // every thread waits for the accumulator: the ring is free after that and becomes the turn-around buffer
+  const bool done = mbar_wait(acc_bar, 0, abort_flag);
+  tc_fence_after();
+  __syncthreads();
+  float *turn = reinterpret_cast<float *>(ring_ptr);          // [128][n_mma + 1] fp32
+  const int ld = p.n_mma + 1;
+  if (done && !s_abort) {
+    if (warp >= 2) {
+      const int quarter = warp & 3;
+      const int r = quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      uint32_t v[32];
+      for (int c0 = 0; c0 < p.n_mma; c0 += 32) {
+        tmem_ld32_issue(taddr + c0, v);
+        tmem_wait_ld();
+        reg_fence32(v);
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (c0 + c < p.n_mma) turn[r * ld + c0 + c] = __uint_as_float(v[c]);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (done && !s_abort) {
+    const int rows = min(kTileM, p.T - row0);
+    const int total = rows * p.n;
+    float *out = p.logits + (size_t)row0 * p.n;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+      const int r = i / p.n, e = i - r * p.n;
+      float v = turn[r * ld + e];
+      if (p.r > 0) {
+        const float *low = turn + r * ld + p.n8;
+        const float *bl = lb_smem ? s_lb + e * p.r : p.lora_b + (size_t)e * p.r;
+        float d = 0.0f;
+        for (int q = 0; q < p.r; ++q) d = fmaf(bl[q], low[q], d);
+        v = fmaf(p.scale, d, v);
+      }
+      out[i] = v;
+    }
+  }
+  // ---------------- teardown ----------------
+  if (s_abort) {
+    if (threadIdx.x == 0 && p.status) atomicCAS(p.status, 0, PCOMOE_ERR_TIMEOUT);
+    const uint64_t t0 = global_ns();
+    for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+  }
+}
+
+// Plain kernel for fp32 layers and shapes the tile does not cover: one block per token; the hidden row is staged
+// in shared memory as fp32, warps take the low-rank rows and then the experts in turn, lanes stride over H.
+template <typename TIn>
+__device__ __forceinline__ float to_f32(TIn v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename TIn>
+__global__ void __launch_bounds__(128) router_simt_kernel(const TIn *h, const TIn *w, const TIn *la, const float *lb,
+                                                          float *logits, int T, int H, int n, int r, float scale) {
+  extern __shared__ float s_row[];      // [H] hidden row, then [r] low-rank activations
+  pdl_grid_wait();
+  float *low = s_row + H;
+  const int t = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+  for (int k = threadIdx.x; k < H; k += blockDim.x) s_row[k] = to_f32<TIn>(h[(size_t)t * H + k]);
+  __syncthreads();
+  for (int q = warp; q < r; q += warps) {
+    float acc = 0.0f;
+    for (int k = lane; k < H; k += 32) acc = fmaf(to_f32<TIn>(la[(size_t)q * H + k]), s_row[k], acc);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) low[q] = acc;
+  }
+  __syncthreads();
+  for (int e = warp; e < n; e += warps) {
+    float acc = 0.0f;
+    for (int k = lane; k < H; k += 32) acc = fmaf(to_f32<TIn>(w[(size_t)e * H + k]), s_row[k], acc);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) {
+      float d = 0.0f;
+      for (int q = 0; q < r; ++q) d = fmaf(lb[(size_t)e * r + q], low[q], d);
+      logits[(size_t)t * n + e] = fmaf(scale, d, acc);
+    }
+  }
+}
+
+}  // namespace
+
+pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, const void *w_router,
+                            const void *lora_a, const float *lora_b, int32_t r, float scale, float *logits,
+                            int32_t *status, cudaStream_t st) {
+  const pcomoe_config &c = L->cfg;
+  const int n = c.n_experts, H = c.hidden;
+  if (status) PCOMOE_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+  const int n8 = (n + 7) & ~7;
+  const int n_mma = (n8 + r + 15) & ~15;
+  const bool tc = c.in_dtype == PCOMOE_BF16 && c.ffn_impl != PCOMOE_FFN_SIMT && H % 8 == 0 && H >= BK &&
+                  n_mma <= 256 && r <= 64;
+  if (tc) {
+    CUtensorMap mH, mW, mL;
+    bool ok = make_map(&mH, h, (uint64_t)T, H, kTileM) && make_map(&mW, w_router, (uint64_t)n, H, (uint32_t)n);
+    if (ok && r > 0) ok = make_map(&mL, lora_a, (uint64_t)r, H, (uint32_t)r);
+    if (!ok) return PCOMOE_ERR_CUDA;
+    if (r == 0) mL = mW;
+    RouterParams p{};
+    p.logits = logits; p.lora_b = lora_b; p.status = status;
+    p.T = T; p.n = n; p.r = r; p.n8 = n8; p.n_mma = n_mma; p.kb = (H + BK - 1) / BK;
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)n_mma >> 3) << 17) | ((128u >> 4) << 24);
+    p.tmem_cols = n_mma <= 32 ? 32u : n_mma <= 64 ? 64u : n_mma <= 128 ? 128u : 256u;
+    p.scale = scale;
+    static bool attr_done = false;
+    if (!attr_done) {
+      PCOMOE_CUDA_TRY(cudaFuncSetAttribute(router_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRSmem));
+      attr_done = true;
+    }
+    PCOMOE_CUDA_TRY(launch_pdl(router_gemm_kernel, dim3((T + kTileM - 1) / kTileM), dim3(kRThreads), kRSmem, st,
+                               mH, mW, mL, p));
+  } else {
+    const size_t smem = sizeof(float) * ((size_t)H + (r > 0 ? r : 1));
+    if (smem > 200 * 1024) return PCOMOE_ERR_UNSUPPORTED;
+    if (c.in_dtype == PCOMOE_BF16) {
+      auto k = router_simt_kernel<__nv_bfloat16>;
+      if (smem > 48 * 1024) PCOMOE_CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      PCOMOE_CUDA_TRY(launch_pdl(k, dim3(T), dim3(128), smem, st, (const __nv_bfloat16 *)h, (const __nv_bfloat16 *)w_router,
+                                 (const __nv_bfloat16 *)lora_a, lora_b, logits, (int)T, H, n, (int)r, scale));
+    } else {
+      auto k = router_simt_kernel<float>;
+      if (smem > 48 * 1024) PCOMOE_CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      PCOMOE_CUDA_TRY(launch_pdl(k, dim3(T), dim3(128), smem, st, (const float *)h, (const float *)w_router,
+                                 (const float *)lora_a, lora_b, logits, (int)T, H, n, (int)r, scale));
+    }
+  }
+  count_launch(status ? 2 : 1);
+  PCOMOE_CUDA_TRY(cudaGetLastError());
+  return PCOMOE_OK;
+}
+
+}  // namespace pcomoe
