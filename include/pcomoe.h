@@ -120,7 +120,8 @@ pcomoe_status pcomoe_layer_active_set(const pcomoe_layer *layer, int32_t cap, in
                                       int32_t *h_tgt, float *h_bias, int32_t *count);
 
 /* Bytes of device workspace pcomoe_build_path_groups and pcomoe_ffn_forward need for up to
- * max_tokens tokens.  The workspace must be 256-byte aligned. */
+ * max_tokens tokens.  The workspace must be 256-byte aligned, and its first 256 bytes (the status words) must
+ * be zero before the first call that uses it; the rest may hold anything. */
 pcomoe_status pcomoe_workspace_bytes(const pcomoe_layer *layer, int32_t max_tokens, size_t *bytes);
 
 /*

@@ -252,6 +252,7 @@ class PathMoELayer:
         self.max_tokens = max_tokens
         self.workspace = torch.empty(pcomoe_workspace_bytes(self.layer, max_tokens), dtype=torch.uint8,
                                      device=self.device)
+        self.workspace[:256].zero_()          # the status words start from zero
         assert self.workspace.data_ptr() % 256 == 0
         T = max(max_tokens, 1)
         self.path_src = torch.zeros(T, top_k, dtype=torch.int32, device=self.device)

@@ -8,6 +8,12 @@ from paper_2609_01024_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
+
+@pytest.fixture(scope="module")
+def G():
+    import gpu_common
+    return gpu_common
+
 # fp32 accumulation of exact bf16 products over H terms, chained over H/16 tensor-core steps: error stays below
 # a few 1e-5 of the sum of magnitudes; the bar below leaves an order of magnitude.
 ABS_TOL, REL_TOL = 1e-3, 1e-3
