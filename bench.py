@@ -287,7 +287,7 @@ def main():
     assert layer.device_status() == 0, "device reported an error during warm-up"
     if args.profile:
         for _ in range(args.steps):
-            layer.forward(d_logits, d_h)
+            step()
         torch.cuda.synchronize()
         print(json.dumps({"profile_run": cfg.name, "steps": args.steps, "status": layer.device_status()}))
         return

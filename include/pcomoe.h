@@ -249,8 +249,8 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, co
  *   d_h        [T,H]  in_dtype, device          d_w_router [n,H]  in_dtype, device
  *   d_lora_a   [r,H]  in_dtype, device or NULL  d_lora_b   [n,r]  fp32, device or NULL   (both when r > 0)
  *   d_logits   [T,n]  fp32, device, written     lora_rank  r >= 0 (0: no adaptation)
- * Products are exact in fp32 (bf16 inputs) and summed in fp32; one thread block owns a tile of 128 tokens from
- * start to end, so the logits are the same bits on every call.  bf16 layers with H % 8 == 0, H >= 64 and
+ * Products are exact in fp32 (bf16 inputs) and summed in fp32 in an order fixed by T and the shapes (no atomics),
+ * so the logits are the same bits on every call with the same T.  bf16 layers with H % 8 == 0, H >= 64 and
  * (n rounded up to 8) + r <= 256, r <= 64 run on the tensor cores; everything else takes a plain kernel.
  * Asynchronous on `stream`; allocates nothing.  The workspace only receives the router's device status word
  * (a wait that ran out -> TIMEOUT), which this call clears first and pcomoe_device_status reports.

@@ -2,12 +2,14 @@
 // scores; Sec. 4.2 calls them the base routing signal g_base(h)):
 //     logits[t,e] = sum_k h[t,k] W_r[e,k]   (+ scale * sum_q B_l[e,q] * sum_k A_l[q,k] h[t,k], the rank-r gate
 //                                              adaptation of Sec. 5.1)
-// The work is a skinny GEMM bound by one read of h, so a tile is 128 tokens x all experts: one CTA streams its
-// 128 rows of h through a 4-stage TMA ring while W_r (and A_l, stacked under it as extra output columns) comes
-// from L2, one thread issues tcgen05.mma (M 128, N = padded n + r, bf16 in, fp32 accumulate in TMEM), and the
-// epilogue turns the accumulators around through shared memory, applies the low-rank term and writes fp32
-// logits coalesced.  One CTA owns a tile from start to end (no split-K, no atomics): logits are reproducible
-// bit for bit, which matters because they decide the TopK.
+// The work is a skinny GEMM bound by one read of h, so a tile is 128 tokens x all experts: a CTA streams rows of
+// h through a deep TMA ring (a stage is 16 KB of h plus the few weight rows, so up to 12 stages are in flight)
+// while W_r (and A_l, stacked under it as extra output columns) comes from L2, one thread issues tcgen05.mma
+// (M 128, N = padded n + r, bf16 in, fp32 accumulate in TMEM), and the epilogue turns the accumulators around
+// through shared memory, applies the low-rank term and writes fp32 logits coalesced.  When the batch has few
+// tiles, a cluster of 2, 4 or 8 CTAs shares each tile along K and adds the partial sums through distributed
+// shared memory in rank order: no atomics, so for a given batch size the logits are reproducible bit for bit,
+// which matters because they decide the TopK.
 // Layers that are not bf16 (or whose shapes the tile does not cover) take a plain SIMT kernel.
 #include <cuda_bf16.h>
 
@@ -16,11 +18,9 @@
 namespace pcomoe {
 namespace {
 
-constexpr int kRStages = 4;
+constexpr int kRMaxStages = 12;
 constexpr uint32_t kRA = kTileM * BK * 2;            // 16 KB of h per k-block
-constexpr uint32_t kRB = 256 * BK * 2;               // up to 256 stacked weight rows per k-block
-constexpr uint32_t kRStage = kRA + kRB;
-constexpr size_t kRSmem = (size_t)kRStages * kRStage + 1024;
+constexpr size_t kRSmem = 196 * 1024 + 1024;         // ring (and, after the MMAs, the turn-around buffers)
 constexpr int kRThreads = 192;
 
 struct RouterParams {
@@ -30,6 +30,9 @@ struct RouterParams {
   int32_t T, n, r, n8;    // n8: row of the stacked tile where A_l starts (n rounded up to 8)
   int32_t n_mma;          // MMA N: n8 + r rounded up to 16
   int32_t kb;             // k-blocks
+  int32_t split;          // CTAs of a cluster that share one tile, each taking a slice of the k-blocks
+  int32_t stages;         // ring depth
+  uint32_t stage_bytes;   // kRA + n_mma * 128
   uint32_t idesc, tmem_cols;
   float scale;
 };
@@ -43,36 +46,59 @@ __device__ __forceinline__ void umma_bf16_n(uint32_t d_tmem, uint64_t adesc, uin
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+__device__ __forceinline__ uint32_t rank_in_cluster() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// fp32 word at shared-memory address `local_addr` of the cluster's CTA `rank`
+__device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+  return v;
+}
 
+// A cluster of `split` CTAs owns one tile of 128 tokens; CTA c of the cluster multiplies k-blocks
+// [c*kb/split, (c+1)*kb/split) and the partial accumulators are added through distributed shared memory in
+// rank order, so the sum does not depend on timing.
 __global__ void __launch_bounds__(kRThreads, 1)
 router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
                    const __grid_constant__ CUtensorMap tmL, const RouterParams p) {
   extern __shared__ unsigned char smem_dyn[];
   pdl_grid_wait();
-  __shared__ __align__(8) uint64_t s_bar[2 * kRStages + 1];
+  __shared__ __align__(8) uint64_t s_bar[2 * kRMaxStages + 1];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ float s_lb[64 * 64];                      // B_l when it fits (n*r <= 4096), else read from global
+  __shared__ float s_lb[64 * 64];                      // B_l transposed to [r][n] when it fits (n*r <= 4096), else global
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char *ring_ptr = smem_dyn + (ring - smem_u32(smem_dyn));
   const uint32_t bar0 = smem_u32(s_bar);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (kRStages + s); };
-  const uint32_t acc_bar = bar0 + 8u * (2 * kRStages);
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kRMaxStages + s); };
+  const uint32_t acc_bar = bar0 + 8u * (2 * kRMaxStages);
   const bool lb_smem = p.r > 0 && p.n * p.r <= 64 * 64;
+  const int crank = p.split > 1 ? (int)rank_in_cluster() : 0;
+  const int tile = blockIdx.x / p.split;
+  const int kb_lo = (int)((int64_t)crank * p.kb / p.split), kb_hi = (int)((int64_t)(crank + 1) * p.kb / p.split);
 
   // rows of the stacked weight tile that no load writes (padding up to the MMA's N) start as zeros
-  for (int s = 0; s < kRStages; ++s) {
-    uint4 *b = reinterpret_cast<uint4 *>(ring_ptr + (size_t)s * kRStage + kRA);
+  for (int s = 0; s < p.stages; ++s) {
+    uint4 *b = reinterpret_cast<uint4 *>(ring_ptr + (size_t)s * p.stage_bytes + kRA);
     for (int i = threadIdx.x; i < p.n_mma * 8; i += blockDim.x) b[i] = make_uint4(0, 0, 0, 0);
   }
   if (lb_smem)
-    for (int i = threadIdx.x; i < p.n * p.r; i += blockDim.x) s_lb[i] = p.lora_b[i];
+    for (int i = threadIdx.x; i < p.n * p.r; i += blockDim.x) s_lb[(i % p.r) * p.n + i / p.r] = p.lora_b[i];
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int s = 0; s < kRStages; ++s) {
+    for (int s = 0; s < p.stages; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
@@ -89,21 +115,21 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = s_tmem;
   volatile int *abort_flag = &s_abort;
-  const int row0 = blockIdx.x * kTileM;
+  const int row0 = tile * kTileM;
   const uint32_t stage_tx = kRA + (uint32_t)(p.n + p.r) * (BK * 2);
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      for (int kb = 0; kb < p.kb; ++kb) {
+      for (int kb = kb_lo; kb < kb_hi; ++kb) {
         if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
-        const uint32_t sa = ring + stage * kRStage, sb = sa + kRA;
+        const uint32_t sa = ring + stage * p.stage_bytes, sb = sa + kRA;
         mbar_arrive_expect_tx(full_bar(stage), stage_tx);
         tma_load_2d(sa, &tmH, kb * BK, row0, full_bar(stage));
         tma_load_2d(sb, &tmW, kb * BK, 0, full_bar(stage));
         if (p.r > 0) tma_load_2d(sb + (uint32_t)p.n8 * (BK * 2), &tmL, kb * BK, 0, full_bar(stage));
-        if (++stage == kRStages) { stage = 0; phase ^= 1u; }
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
     }
     __syncwarp();
@@ -112,16 +138,16 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int kb = 0; kb < p.kb; ++kb) {
+      for (int kb = kb_lo; kb < kb_hi; ++kb) {
         if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t sa = ring + stage * kRStage, sb = sa + kRA;
+        const uint32_t sa = ring + stage * p.stage_bytes, sb = sa + kRA;
         const uint64_t da = umma_desc(sa), db = umma_desc(sb);
 #pragma unroll
         for (int k = 0; k < BK / 16; ++k)
-          umma_bf16_n(tmem_base, da + 2u * k, db + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_bf16_n(tmem_base, da + 2u * k, db + 2u * k, p.idesc, (kb > kb_lo || k != 0) ? 1u : 0u);
         umma_commit(empty_bar(stage));
-        if (++stage == kRStages) { stage = 0; phase ^= 1u; }
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
       if (alive) umma_commit(acc_bar);
     }
@@ -131,7 +157,7 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   const bool done = mbar_wait(acc_bar, 0, abort_flag);
   tc_fence_after();
   __syncthreads();
-  float *turn = reinterpret_cast<float *>(ring_ptr);          // [128][n_mma + 1] fp32
+  float *turn = reinterpret_cast<float *>(ring_ptr);          // [128][n_mma + 1] fp32: this CTA's partial sums
   const int ld = p.n_mma + 1;
   if (done && !s_abort) {
     if (warp >= 2) {
@@ -151,23 +177,47 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   }
   tc_fence_before();
   __syncthreads();
+  // rows of the tile this CTA finishes: an equal share per CTA of the cluster
+  const int share = kTileM / p.split;
+  const int r_lo = crank * share;
+  const float *sums = turn;                                   // [.][ld], indexed by tile row
+  if (p.split > 1) {
+    cluster_barrier();                                        // every CTA's partial sums are in place
+    float *red = turn + kTileM * ld;                          // [share][ld]: the cluster's sums for this CTA's rows
+    const uint32_t turn_addr = ring;
+    for (int i = threadIdx.x; i < share * p.n_mma; i += blockDim.x) {
+      const int rr = i / p.n_mma, c = i - rr * p.n_mma;
+      const uint32_t off = (uint32_t)(((r_lo + rr) * ld + c) * 4);
+      float acc = 0.0f;
+      for (int s = 0; s < p.split; ++s) acc += ld_peer_f32(turn_addr + off, (uint32_t)s);
+      red[rr * ld + c] = acc;
+    }
+    __syncthreads();
+    sums = red - r_lo * ld;                                   // so that sums[r * ld + c] addresses tile row r
+  }
   if (done && !s_abort) {
     const int rows = min(kTileM, p.T - row0);
-    const int total = rows * p.n;
-    float *out = p.logits + (size_t)row0 * p.n;
+    const int r_hi = min(rows, r_lo + share);
+    const int total = (r_hi - r_lo) * p.n;
+    float *out = p.logits + ((size_t)row0 + r_lo) * p.n;
     for (int i = threadIdx.x; i < total; i += blockDim.x) {
-      const int r = i / p.n, e = i - r * p.n;
-      float v = turn[r * ld + e];
+      const int r = r_lo + i / p.n, e = i % p.n;
+      float v = sums[r * ld + e];
       if (p.r > 0) {
-        const float *low = turn + r * ld + p.n8;
-        const float *bl = lb_smem ? s_lb + e * p.r : p.lora_b + (size_t)e * p.r;
+        const float *low = sums + r * ld + p.n8;
         float d = 0.0f;
-        for (int q = 0; q < p.r; ++q) d = fmaf(bl[q], low[q], d);
+        if (lb_smem) {   // neighbouring threads hold neighbouring experts: [r][n] keeps their reads on separate banks
+          for (int q = 0; q < p.r; ++q) d = fmaf(s_lb[q * p.n + e], low[q], d);
+        } else {
+          const float *bl = p.lora_b + (size_t)e * p.r;
+          for (int q = 0; q < p.r; ++q) d = fmaf(bl[q], low[q], d);
+        }
         v = fmaf(p.scale, d, v);
       }
       out[i] = v;
     }
   }
+  if (p.split > 1) cluster_barrier();                         // peers may still be reading this CTA's sums
   // ---------------- teardown ----------------
   if (s_abort) {
     if (threadIdx.x == 0 && p.status) atomicCAS(p.status, 0, PCOMOE_ERR_TIMEOUT);
@@ -245,13 +295,35 @@ pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, con
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)n_mma >> 3) << 17) | ((128u >> 4) << 24);
     p.tmem_cols = n_mma <= 32 ? 32u : n_mma <= 64 ? 64u : n_mma <= 128 ? 128u : 256u;
     p.scale = scale;
+    p.stage_bytes = kRA + (uint32_t)n_mma * (BK * 2);
+    p.stages = (int)((kRSmem - 1024) / p.stage_bytes);
+    if (p.stages > kRMaxStages) p.stages = kRMaxStages;
+    // few tiles: a cluster shares each tile along K so that more SMs stream h (powers of two up to 8, at least
+    // two k-blocks per CTA, and only while the partial sums of a cluster fit next to the reduced rows)
+    const int tiles = (T + kTileM - 1) / kTileM;
+    int split = 1;
+    while (split < 8 && tiles * split * 2 <= L->sm_count && p.kb >= 4 * split && n_mma <= 128) split *= 2;
+    p.split = split;
     static bool attr_done = false;
     if (!attr_done) {
       PCOMOE_CUDA_TRY(cudaFuncSetAttribute(router_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRSmem));
       attr_done = true;
     }
-    PCOMOE_CUDA_TRY(launch_pdl(router_gemm_kernel, dim3((T + kTileM - 1) / kTileM), dim3(kRThreads), kRSmem, st,
-                               mH, mW, mL, p));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles * split);
+    cfg.blockDim = dim3(kRThreads);
+    cfg.dynamicSmemBytes = kRSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = split;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = split > 1 ? 2 : 1;
+    PCOMOE_CUDA_TRY(cudaLaunchKernelEx(&cfg, router_gemm_kernel, mH, mW, mL, p));
   } else {
     const size_t smem = sizeof(float) * ((size_t)H + (r > 0 ? r : 1));
     if (smem > 200 * 1024) return PCOMOE_ERR_UNSUPPORTED;
