@@ -253,7 +253,7 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, co
  * so the logits are the same bits on every call with the same T.  bf16 layers with H % 8 == 0, H >= 64 and
  * (n rounded up to 8) + r <= 256, r <= 64 run on the tensor cores; everything else takes a plain kernel.
  * Asynchronous on `stream`; allocates nothing.  The workspace only receives the router's device status word
- * (a wait that ran out -> TIMEOUT), which this call clears first and pcomoe_device_status reports.
+ * (a wait that ran out -> TIMEOUT), which stays set until pcomoe_device_status has reported it.
  * Errors: INVALID_ARG (NULL pointers, r < 0), SHAPE (T < 0, r > 256), WORKSPACE, UNSUPPORTED (plain kernel:
  * H too large for shared memory), CUDA. */
 pcomoe_status pcomoe_router_logits(const pcomoe_layer *layer, int32_t T, const void *d_h,
@@ -261,9 +261,18 @@ pcomoe_status pcomoe_router_logits(const pcomoe_layer *layer, int32_t T, const v
                                    int32_t lora_rank, float lora_scale, float *d_logits, void *d_workspace,
                                    size_t ws_bytes, void *stream);
 
+/* Residual stream between the layers of a multi-layer loop (the paper's layer output y of Sec. 4.1 is added to the
+ * block's input, as in any transformer block; the paper does not write this step out): 
+ *     d_h_out[t,k] = round(d_h_in[t,k] + d_y[t,k])
+ * one fp32 addition per element, rounded to nearest-even into the layer's storage type (exact copy of the sum
+ * for fp32 layers).  d_h_in, d_h_out [T,H] in_dtype (may be the same array); d_y [T,H] fp32.  Asynchronous on
+ * `stream`; allocates nothing.  Errors: INVALID_ARG, SHAPE (T < 0), CUDA. */
+pcomoe_status pcomoe_residual_cast(const pcomoe_layer *layer, int32_t T, const void *d_h_in, const float *d_y,
+                                   void *d_h_out, void *stream);
+
 /* Synchronises `stream`, reads the workspace's status words and returns the first error a kernel
  * recorded (PCOMOE_OK if none): the layer's word is cleared by the next pcomoe_build_path_groups, the
- * router's by the next pcomoe_router_logits. */
+ * router's by this call once it has been read. */
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream);
 
 /* Launch counters (kernels and memsets enqueued by this library since load, per process). */

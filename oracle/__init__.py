@@ -206,3 +206,17 @@ def router_logits(h, w_router, lora_a=None, lora_b=None, lora_scale=1.0):
     if rc != 0:
         raise ValueError(f"pcomoe_oracle_router_logits failed with code {rc}")
     return out
+
+
+def residual_cast(h_in, y):
+    """h_out = round(h_in + y): fp32 add, then bf16 round-to-nearest-even when ``h_in`` is bf16 bit patterns
+    (uint16), else the fp32 sum."""
+    h = np.ascontiguousarray(h_in)
+    yy = _c(y, np.float32)
+    assert h.shape == yy.shape
+    out = np.empty_like(h)
+    rc = _load().pcomoe_oracle_residual_cast(ctypes.c_int64(h.size), _p(h), _p(yy), _p(out),
+                                             ctypes.c_int32(_wdtype(h)))
+    if rc != 0:
+        raise ValueError(f"pcomoe_oracle_residual_cast failed with code {rc}")
+    return out

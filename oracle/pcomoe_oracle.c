@@ -408,3 +408,41 @@ int pcomoe_oracle_mask_tighten(int32_t n, const float *B, const uint8_t *M_prev,
   }
   return ORACLE_OK;
 }
+
+/* ---------------------------------------------------------------------------
+ * Residual stream between layers of a multi-layer loop: h_out = round(h_in + y).  The result is the next
+ * layer's stored input (a quantised code when the storage type is bf16), so the precision of the decision is
+ * fixed here as the CUDA path fixes it: one fp32 addition, then round-to-nearest-even to bf16 (wdtype = bf16;
+ * the bf16 values travel as bit patterns) or the fp32 sum itself (wdtype = fp32).  The paper does not write
+ * this step out; it is the usual residual connection around the block whose output is y (Sec. 4.1).
+ * ------------------------------------------------------------------------- */
+static uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); /* NaN stays NaN */
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7fffu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+int pcomoe_oracle_residual_cast(int64_t count, const void *h_in, const float *y, void *h_out, int32_t wdtype) {
+  if (count < 0 || !h_in || !y || !h_out) return ORACLE_ERR_ARG;
+  if (wdtype == ORACLE_W_F32) {
+    const float *a = (const float *)h_in;
+    float *o = (float *)h_out;
+    for (int64_t i = 0; i < count; ++i) {
+      volatile float s = a[i] + y[i];
+      o[i] = s;
+    }
+  } else if (wdtype == ORACLE_W_BF16) {
+    const uint16_t *a = (const uint16_t *)h_in;
+    uint16_t *o = (uint16_t *)h_out;
+    for (int64_t i = 0; i < count; ++i) {
+      volatile float s = bf16_bits_to_f32(a[i]) + y[i];
+      o[i] = f32_to_bf16_rne(s);
+    }
+  } else {
+    return ORACLE_ERR_ARG;
+  }
+  return ORACLE_OK;
+}

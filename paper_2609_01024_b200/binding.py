@@ -22,7 +22,7 @@ PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR = 
 
 EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_mask_tighten", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
            "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",
-           "pcomoe_ffn_forward_stages", "pcomoe_router_logits",
+           "pcomoe_ffn_forward_stages", "pcomoe_router_logits", "pcomoe_residual_cast",
            "pcomoe_device_status",
            "pcomoe_launch_count", "pcomoe_status_string"]
 
@@ -71,6 +71,7 @@ def load_library(path: str | None = None):
     lib.pcomoe_ffn_forward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
     lib.pcomoe_ffn_forward_stages.argtypes = lib.pcomoe_ffn_forward.argtypes + [i32]
     lib.pcomoe_router_logits.argtypes = [vp, i32, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, sz, vp]
+    lib.pcomoe_residual_cast.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.pcomoe_device_status.argtypes = [vp, vp]
     lib.pcomoe_launch_count.restype = ctypes.c_int64
     lib.pcomoe_status_string.restype = ctypes.c_char_p
@@ -227,6 +228,11 @@ def pcomoe_router_logits(layer, T, h, w_router, lora_a, lora_b, lora_rank: int, 
                                                lora_rank, lora_scale, _ptr(logits), _ptr(workspace),
                                                workspace.numel() * workspace.element_size(), _stream()),
            "pcomoe_router_logits")
+
+
+def pcomoe_residual_cast(layer, T, h_in, y, h_out):
+    _check(load_library().pcomoe_residual_cast(layer, T, _ptr(h_in), _ptr(y), _ptr(h_out), _stream()),
+           "pcomoe_residual_cast")
 
 
 def pcomoe_device_status(workspace) -> int:
@@ -398,6 +404,47 @@ class PathMoELayer:
 
     def device_status(self) -> int:
         return pcomoe_device_status(self.workspace)
+
+
+class PathMoEStack:
+    """A decode-step loop over several path-composed MoE blocks, each with its own mask, bias, router and expert
+    weights: per block  router -> route -> group -> stage 1 -> stage 2 -> residual, the hidden states staying on
+    the device in the layers' storage type.  `capture()` records the whole step into one CUDA graph.
+    Marshalling only: every step runs in the library's kernels."""
+
+    def __init__(self, layers):
+        assert layers and all(getattr(l, "w_router", None) is not None for l in layers), "every block needs set_router()"
+        self.layers = list(layers)
+        l0 = self.layers[0]
+        self.device, self.H, self.max_tokens = l0.device, l0.H, min(l.max_tokens for l in self.layers)
+        dt = l0.w_router.dtype
+        # hidden states entering every block, and leaving the last one
+        self.h = [torch.empty(self.max_tokens, self.H, dtype=dt, device=self.device) for _ in range(len(layers) + 1)]
+
+    def decode_step(self, h):
+        """h [T,H] device tensor in the storage type -> hidden states after the last block (a view of an internal
+        buffer).  The per-block inputs stay readable in `self.h[l][:T]`."""
+        T = h.shape[0]
+        assert T <= self.max_tokens
+        self.h[0][:T].copy_(h)
+        for l, layer in enumerate(self.layers):
+            layer.forward_hidden(self.h[l][:T])
+            pcomoe_residual_cast(layer.layer, T, self.h[l], layer.y, self.h[l + 1])
+        return self.h[-1][:T]
+
+    def capture(self, h):
+        """Graph of one decode step reading `h` (fixed device tensor).  Call decode_step once before capturing."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.decode_step(h)
+        return g
+
+    def device_status(self) -> int:
+        for layer in self.layers:
+            st = layer.device_status()
+            if st:
+                return st
+        return 0
 
 
 def to_device(arr: np.ndarray | None, device="cuda:0"):

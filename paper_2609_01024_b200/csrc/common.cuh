@@ -122,6 +122,8 @@ pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, con
 pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, const void *w_router,
                             const void *lora_a, const float *lora_b, int32_t r, float scale, float *logits,
                             int32_t *status, cudaStream_t st);
+pcomoe_status launch_residual_cast(const pcomoe_layer *L, int32_t T, const void *h_in, const float *y, void *h_out,
+                                   cudaStream_t st);
 pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src, const int32_t *tgt,
                             const float *w, const pcomoe_groups *g, char *ws, const WsLayout &lay,
                             cudaStream_t st);

@@ -1,4 +1,5 @@
 // Host side of the C ABI: layer set-up, workspace sizing, argument checks and dispatch.
+#include <cstddef>
 #include <algorithm>
 #include <atomic>
 #include <cmath>
@@ -274,6 +275,15 @@ pcomoe_status pcomoe_router_logits(const pcomoe_layer *L, int32_t T, const void 
                        &plan->status_router, (cudaStream_t)stream);
 }
 
+pcomoe_status pcomoe_residual_cast(const pcomoe_layer *L, int32_t T, const void *d_h_in, const float *d_y,
+                                   void *d_h_out, void *stream) {
+  if (!L) return PCOMOE_ERR_INVALID_ARG;
+  if (T < 0) return PCOMOE_ERR_SHAPE;
+  if (T == 0) return PCOMOE_OK;
+  if (!d_h_in || !d_y || !d_h_out) return PCOMOE_ERR_INVALID_ARG;
+  return launch_residual_cast(L, T, d_h_in, d_y, d_h_out, (cudaStream_t)stream);
+}
+
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream) {
   if (!d_workspace) return PCOMOE_ERR_WORKSPACE;
   DevPlan plan;
@@ -281,6 +291,11 @@ pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream) {
   if (cudaMemcpy(&plan, d_workspace, sizeof(DevPlan), cudaMemcpyDeviceToHost) != cudaSuccess)
     return PCOMOE_ERR_CUDA;
   const int32_t st = plan.status ? plan.status : plan.status_router;
+  if (plan.status_router != 0) {   // the router's word is sticky: reading it clears it
+    if (cudaMemset((char *)const_cast<void *>(d_workspace) + offsetof(DevPlan, status_router), 0, sizeof(int32_t)) !=
+        cudaSuccess)
+      return PCOMOE_ERR_CUDA;
+  }
   if (st < 0 || st > PCOMOE_ERR_INDEX) return PCOMOE_ERR_CUDA;
   return (pcomoe_status)st;
 }

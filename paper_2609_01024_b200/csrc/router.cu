@@ -278,7 +278,6 @@ pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, con
                             int32_t *status, cudaStream_t st) {
   const pcomoe_config &c = L->cfg;
   const int n = c.n_experts, H = c.hidden;
-  if (status) PCOMOE_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
   const int n8 = (n + 7) & ~7;
   const int n_mma = (n8 + r + 15) & ~15;
   const bool tc = c.in_dtype == PCOMOE_BF16 && c.ffn_impl != PCOMOE_FFN_SIMT && H % 8 == 0 && H >= BK &&
@@ -339,7 +338,7 @@ pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, con
                                  (const float *)lora_a, lora_b, logits, (int)T, H, n, (int)r, scale));
     }
   }
-  count_launch(status ? 2 : 1);
+  count_launch();
   PCOMOE_CUDA_TRY(cudaGetLastError());
   return PCOMOE_OK;
 }

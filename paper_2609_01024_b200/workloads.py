@@ -216,6 +216,14 @@ def small_case(seed: int, T: int, H: int, F: int, n: int, K: int, mask_p: float 
                        mask_p=mask_p, F_sh=F_sh, dtype=dtype, logits=logits, zipf_a=zipf_a, lam=lam)
 
 
+def stack_layer_config(cfg: LayerConfig, l: int, native_blocks: int = 2) -> LayerConfig:
+    """Config of block ``l`` of a multi-layer stack built on ``cfg``: its own seed (mask, bias, router and expert
+    weights differ per block) and its own path density - the first ``native_blocks`` blocks keep every path
+    active, pruning applies from the next block on (Sec. 5.3, pruning sensitivity)."""
+    return cfg.scaled(name=f"{cfg.name}-block{l}", seed=cfg.seed + 1000 * (l + 1),
+                      mask_p=1.0 if l < native_blocks else cfg.mask_p)
+
+
 @dataclasses.dataclass
 class LayerInputs:
     cfg: LayerConfig
