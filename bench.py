@@ -199,6 +199,92 @@ def run_reference(args, cfg):
     print(json.dumps(out), flush=True)
 
 
+def run_stack(args, cfg, L, layer0, d_h, dev, rank, world, stream):
+    """Decode step through `--layers` blocks.  Every block has its own mask, bias and router (seeded per block; the
+    first two keep every path, Sec. 5.3) and its own copy of the expert weights in HBM, so that every step streams
+    L distinct weight sets; the copies hold the same seeded values (drawing L x 2.8 GB on the host would take
+    minutes and changes nothing that is timed)."""
+    import torch
+    from paper_2609_01024_b200 import binding as B
+    dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
+    blocks = []
+    for l in range(args.layers):
+        c = wl.stack_layer_config(cfg, l)
+        wts = (layer0.w_gate, layer0.w_up, layer0.w_down) if l == 0 else tuple(x.clone() for x in (layer0.w_gate, layer0.w_up, layer0.w_down))
+        shared = None
+        if cfg.F_sh:
+            shared = layer0.shared if l == 0 else tuple(x.clone() for x in layer0.shared)
+        blk = layer0 if l == 0 else None
+        blk = B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=cfg.F, mask=wl.make_mask(c), bias=wl.make_bias(c),
+                             w_gate=wts[0], w_up=wts[1], w_down=wts[2], shared=shared, max_tokens=cfg.T, in_dtype=dt,
+                             lam=cfg.lam, ffn_impl=args.ffn_impl, device=dev)
+        w_r, l_a, l_b = wl.make_router_weights(c, lora_rank=max(args.router, 0))
+        blk.set_router(B.to_device(w_r, dev), B.to_device(l_a, dev), None if l_b is None else torch.from_numpy(l_b).to(dev), 1.0)
+        blocks.append(blk)
+    stack = B.PathMoEStack(blocks)
+    stack.decode_step(d_h)
+    torch.cuda.synchronize()
+    m0 = B.pcomoe_launch_count(); stack.decode_step(d_h); per_step = B.pcomoe_launch_count() - m0
+    torch.cuda.synchronize()
+    graph = stack.capture(d_h)
+    for _ in range(args.warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert stack.device_status() == 0
+    try:
+        uuid = torch.cuda.get_device_properties(dev).uuid
+    except Exception:
+        uuid = None
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")), uuid)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    assert stack.device_status() == 0
+    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+    # end to end: hidden states from pinned host memory, final hidden states back to the host
+    pin_h = (torch.from_numpy(L.h.view(np.int16)).view(torch.bfloat16) if L.h.dtype == np.uint16 else torch.from_numpy(L.h)).pin_memory()
+    pin_out = torch.empty_like(pin_h).pin_memory()
+    def host_step():
+        d_h.copy_(pin_h, non_blocking=True)
+        graph.replay()
+        pin_out.copy_(stack.h[-1][:cfg.T], non_blocking=True)
+    for _ in range(3):
+        host_step()
+    torch.cuda.synchronize()
+    tw = time.perf_counter()
+    for _ in range(args.steps):
+        host_step()
+    torch.cuda.synchronize()
+    e2e = world * cfg.T * args.steps / replicas.max_over_ranks(time.perf_counter() - tw, dev)
+    pk = peaks()
+    es = 4 if cfg.dtype == "f32" else 2
+    wbytes = args.layers * es * (3 * cfg.n * cfg.H * cfg.F + 3 * cfg.H * cfg.F_sh)
+    ach = wbytes / (ms * 1e-3) / 1e9
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": replicas.whole_job_tokens_per_s(cfg.T, world, ms), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfg.dtype != "f32" else "f32", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}-x{args.layers}blocks", "T": cfg.T, "H": cfg.H, "F": cfg.F, "n": cfg.n, "K": cfg.K,
+                       "F_sh": cfg.F_sh, "blocks": args.layers, "router_lora_rank": max(args.router, 0), "cuda_graph": True,
+                       "l2": "inputs larger than L2 (every block streams its own weights)",
+                       "note": "a token counts once per step through all blocks"},
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": int(L.h.nbytes), "d2h_bytes_per_step": int(L.h.nbytes)},
+            "gpu_launches": int(per_step * args.steps), "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
+                         "traffic": None, "kernel": "whole step: expert weights of every block streamed once",
+                         "peak_source": pk["source"] + " copy bandwidth"},
+            "ms_per_block": ms / args.layers}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -217,6 +303,9 @@ def main():
     ap.add_argument("--router", type=int, default=-1,
                     help="r >= 0: the timed step starts from hidden states (router GEMM with a rank-r gate adaptation, "
                          "0 = none, in front of the path gate); default -1: logits are an input, as the metric is quoted")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="L > 0: time a decode step through a stack of L blocks (router + path gate + FFN + residual "
+                         "per block, one CUDA graph per step) instead of the single-layer metric")
     ap.add_argument("--graph", action="store_true",
                     help="replay the hot path from a CUDA graph in the device-resident timing loop")
     ap.add_argument("--ffn-impl", type=int, default=0,
@@ -262,6 +351,9 @@ def main():
     d_logits = torch.from_numpy(L.logits).to(dev)
     d_h = B.to_device(L.h, dev)
     stream = torch.cuda.current_stream()
+    if args.layers > 0:
+        run_stack(args, cfg, L, layer, d_h, dev, rank, world, stream)
+        return
 
     def barrier():
         torch.cuda.synchronize()
