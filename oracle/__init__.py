@@ -124,6 +124,33 @@ def groups(src, tgt, w, n, dedup=1):
     return out
 
 
+def groups_target_reuse(src, tgt, w, n, dedup=1):
+    """Group arrays with projection-side reuse: stage 1 as `groups`, stage 2 over unique (token, target) rows.
+    Adds R2, s2_cnt (contributors per row) and path_s2row [T,K]."""
+    g = groups(src, tgt, w, n, dedup=dedup)
+    tgt, w = _c(tgt, np.int32), _c(w, np.float32)
+    T, K = tgt.shape
+    P = T * K
+    out = dict(s2_offsets=np.zeros(n + 1, np.int32), s2_path=np.zeros(max(P, 1), np.int32),
+               s2_s1row=np.zeros(max(P, 1), np.int32), s2_token=np.zeros(max(P, 1), np.int32),
+               s2_w=np.zeros(max(P, 1), np.float32), s2_cnt=np.zeros(max(P, 1), np.int32),
+               path_s2row=np.zeros((T, K), np.int32))
+    r2 = ctypes.c_int32(0)
+    ps1 = np.ascontiguousarray(g["path_s1row"])
+    rc = _load().pcomoe_oracle_groups_target_reuse(ctypes.c_int32(T), ctypes.c_int32(n), ctypes.c_int32(K), _p(tgt),
+                                                   _p(w), _p(ps1), _p(out["s2_offsets"]), _p(out["s2_path"]),
+                                                   _p(out["s2_s1row"]), _p(out["s2_token"]), _p(out["s2_w"]),
+                                                   _p(out["s2_cnt"]), _p(out["path_s2row"]), ctypes.byref(r2))
+    if rc != 0:
+        raise ValueError(f"pcomoe_oracle_groups_target_reuse failed with code {rc}")
+    R2 = int(r2.value)
+    for k in ("s2_path", "s2_s1row", "s2_token", "s2_w", "s2_cnt"):
+        out[k] = out[k][:R2].copy()
+    g.update(out)
+    g["R2"] = R2
+    return g
+
+
 def _wdtype(w):
     if w.dtype == np.float32:
         return W_F32

@@ -189,6 +189,50 @@ int pcomoe_oracle_groups(int32_t T, int32_t n, int32_t K, int32_t dedup, const i
   return ORACLE_OK;
 }
 
+/* ---------------------------------------------------------------------------
+ * Target grouping with projection-side reuse.  D_j is linear, so for one token
+ *   sum_{i in paths with target j} beta_ij D_j(U_i(h)) = D_j( sum_i beta_ij U_i(h) )
+ * (Sec. 3.2 counts what reusing the projection side would save; Sec. 4.1 defines D_j(a) = W_down a).
+ * A stage-2 row is then a unique (token, target):
+ *   path (t,k) is "primary" iff no k' < k of the token has the same target; the others join their primary's row
+ *   stage-2 rows: for j ascending, for primary paths q = t*K+k ascending with tgt = j
+ *   s2_w   = the path's weight when the row has one contributor, 1 when it has several (the weights then
+ *            scale the contributions that are summed into the row)
+ *   s2_cnt = contributors of the row;  path_s2row[q] = the row path q feeds
+ * path_s1row comes from pcomoe_oracle_groups.  Arrays hold T*K entries; R2 rows are written.
+ * ------------------------------------------------------------------------- */
+int pcomoe_oracle_groups_target_reuse(int32_t T, int32_t n, int32_t K, const int32_t *tgt, const float *w,
+                                      const int32_t *path_s1row, int32_t *s2_offsets, int32_t *s2_path,
+                                      int32_t *s2_s1row, int32_t *s2_token, float *s2_w, int32_t *s2_cnt,
+                                      int32_t *path_s2row, int32_t *R2_out) {
+  if (T < 0 || n <= 0 || K <= 0) return ORACLE_ERR_ARG;
+  int32_t r2 = 0;
+  for (int32_t j = 0; j < n; ++j) {
+    s2_offsets[j] = r2;
+    for (int32_t t = 0; t < T; ++t) {
+      int32_t first = -1, cnt = 0;
+      for (int32_t k = 0; k < K; ++k)
+        if (tgt[(size_t)t * K + k] == j) {
+          if (first < 0) first = k;
+          ++cnt;
+        }
+      if (first < 0) continue;
+      const int32_t q = t * K + first;
+      s2_path[r2] = q;
+      s2_s1row[r2] = path_s1row[q];
+      s2_token[r2] = t;
+      s2_w[r2] = cnt == 1 ? w[q] : 1.0f;
+      s2_cnt[r2] = cnt;
+      for (int32_t k = 0; k < K; ++k)
+        if (tgt[(size_t)t * K + k] == j) path_s2row[(size_t)t * K + k] = r2;
+      ++r2;
+    }
+  }
+  s2_offsets[n] = r2;
+  *R2_out = r2;
+  return ORACLE_OK;
+}
+
 /* exact upcast of a bf16 bit pattern */
 static inline float bf16_bits_to_f32(uint16_t b) {
   uint32_t u = (uint32_t)b << 16;
