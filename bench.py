@@ -303,6 +303,8 @@ def main():
     ap.add_argument("--router", type=int, default=-1,
                     help="r >= 0: the timed step starts from hidden states (router GEMM with a rank-r gate adaptation, "
                          "0 = none, in front of the path gate); default -1: logits are an input, as the metric is quoted")
+    ap.add_argument("--target-reuse", type=int, default=0,
+                    help="1: projection-side reuse (one stage-2 row per unique (token, target), exact by linearity)")
     ap.add_argument("--layers", type=int, default=0,
                     help="L > 0: time a decode step through a stack of L blocks (router + path gate + FFN + residual "
                          "per block, one CUDA graph per step) instead of the single-layer metric")
@@ -347,7 +349,8 @@ def main():
                            w_gate=B.to_device(L.w_gate, dev), w_up=B.to_device(L.w_up, dev),
                            w_down=B.to_device(L.w_down, dev),
                            shared=tuple(B.to_device(x, dev) for x in (L.wsh_gate, L.wsh_up, L.wsh_down)) if cfg.F_sh else None,
-                           max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam, ffn_impl=args.ffn_impl, device=dev)
+                           max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam, ffn_impl=args.ffn_impl,
+                           target_reuse=args.target_reuse, device=dev)
     d_logits = torch.from_numpy(L.logits).to(dev)
     d_h = B.to_device(L.h, dev)
     stream = torch.cuda.current_stream()
@@ -476,7 +479,8 @@ def main():
                "vs_baseline": None, "dtype": "bf16" if tc_path else "f32", "data": "synthetic",
                "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
                           "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam,
-                          "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(args.graph),
+                          "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(args.graph), "target_reuse": int(args.target_reuse),
+                          "stage2_rows_over_P": int(stats[1]) / (cfg.T * cfg.K),
                           "router_in_step": (f"yes (rank-{args.router} gate adaptation)" if args.router > 0 else
                                              "yes" if args.router == 0 else "no (logits are an input)"),
                           "parallelism": f"token-dp{world} (replicas, no collective)",

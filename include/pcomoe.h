@@ -72,6 +72,11 @@ typedef struct {
   int32_t dedup;        /* 1: one stage-1 row per unique (token, source)  (Sec. 4.3 reuse);
                            0: one stage-1 row per path                                        */
   int32_t ffn_impl;     /* pcomoe_ffn_impl                                                    */
+  int32_t target_reuse; /* 1: one stage-2 row per unique (token, target): the weighted intermediates of
+                           a token's paths that share a target are summed before the projection, which
+                           is exact by linearity of D_j (Sec. 3.2, 4.1); tensor-core layers only.
+                           0 (default): one stage-2 row per path.  A struct_size that ends before this
+                           field is accepted and means 0.                                     */
 } pcomoe_config;
 
 typedef struct pcomoe_layer pcomoe_layer; /* opaque; owns the small device table of active paths */

@@ -38,7 +38,7 @@ class pcomoe_config(ctypes.Structure):
                 ("hidden", ctypes.c_int32), ("ffn", ctypes.c_int32), ("shared_ffn", ctypes.c_int32),
                 ("in_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32), ("lambda_", ctypes.c_float),
                 ("norm_topk", ctypes.c_int32), ("routed_scale", ctypes.c_float), ("dedup", ctypes.c_int32),
-                ("ffn_impl", ctypes.c_int32)]
+                ("ffn_impl", ctypes.c_int32), ("target_reuse", ctypes.c_int32)]
 
 
 class pcomoe_groups(ctypes.Structure):
@@ -100,10 +100,10 @@ def pcomoe_launch_count() -> int:
 
 def pcomoe_layer_create(*, n_experts, top_k, hidden, ffn, mask, bias, shared_ffn=0, in_dtype=PCOMOE_BF16,
                         out_dtype=PCOMOE_FP32, lam=0.5, norm_topk=1, routed_scale=1.0, dedup=1,
-                        ffn_impl=PCOMOE_FFN_AUTO):
+                        ffn_impl=PCOMOE_FFN_AUTO, target_reuse=0):
     lib = load_library()
     cfg = pcomoe_config(ctypes.sizeof(pcomoe_config), n_experts, top_k, hidden, ffn, shared_ffn, in_dtype,
-                        out_dtype, lam, norm_topk, routed_scale, dedup, ffn_impl)
+                        out_dtype, lam, norm_topk, routed_scale, dedup, ffn_impl, target_reuse)
     m = np.ascontiguousarray(mask, dtype=np.uint8)
     b = np.ascontiguousarray(bias, dtype=np.float32)
     assert m.size == n_experts * n_experts and b.size == n_experts * n_experts
@@ -244,7 +244,7 @@ class PathMoELayer:
 
     def __init__(self, *, n_experts, top_k, hidden, ffn, mask, bias, w_gate, w_up, w_down, shared=None,
                  max_tokens, in_dtype=PCOMOE_BF16, lam=0.5, norm_topk=1, routed_scale=1.0, dedup=1,
-                 ffn_impl=PCOMOE_FFN_AUTO, device="cuda:0"):
+                 ffn_impl=PCOMOE_FFN_AUTO, target_reuse=0, device="cuda:0"):
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self.n, self.K, self.H, self.F = n_experts, top_k, hidden, ffn
@@ -252,7 +252,8 @@ class PathMoELayer:
         self.layer = pcomoe_layer_create(n_experts=n_experts, top_k=top_k, hidden=hidden, ffn=ffn, mask=mask,
                                          bias=bias, shared_ffn=self.F_sh, in_dtype=in_dtype, lam=lam,
                                          norm_topk=norm_topk, routed_scale=routed_scale, dedup=dedup,
-                                         ffn_impl=ffn_impl)
+                                         ffn_impl=ffn_impl, target_reuse=target_reuse)
+        self.target_reuse = int(target_reuse)
         self.w_gate, self.w_up, self.w_down = w_gate, w_up, w_down
         self.shared = shared if self.F_sh else (None, None, None)
         self.max_tokens = max_tokens

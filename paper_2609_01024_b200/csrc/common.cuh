@@ -48,6 +48,7 @@ struct WsLayout {
                        //                            order; SIMT path: by unpadded stage-1 row)
   size_t u_sh;         // in_dtype [Tpad, F_sh]      shared-expert intermediates
   size_t h_gath;       // bf16 [mt_max*128, H]       rows of h in padded stage-1 order (tensor-core path)
+  size_t path_wgt;     // fp32 [T*K]                 copy of the path weights (projection-side reuse only)
   size_t total;
   int32_t nb_max;      // blocks of the grouping kernels at max_tokens
   int32_t mt_max;      // upper bound of m-tiles per stage

@@ -45,7 +45,9 @@ struct Seg {
   // stage 1: where a row's SwiGLU output goes
   const int32_t *row_token;    // token of a padded row (routed), NULL: the row is its own destination
   const int32_t *path_prow1;   // [T,K] padded stage-1 row of every path
-  const int32_t *path_pos2;    // [T,K] padded stage-2 row of every path (= row of u_out to write)
+  const int32_t *path_pos2;    // [T,K] padded stage-2 row of every path (= row of u_out to write); a row that
+                               //       several paths of the token feed is stored as -(row + 2)
+  const float *path_w;         // [T,K] path weights: scale of a contribution to such a shared row
   __nv_bfloat16 *u_out;
   int32_t ldu;
   // stage 2: where a row's projection goes
@@ -127,10 +129,11 @@ struct RowCtx {
   int my_prow;        // padded row of this thread
   int nd;             // stage 1, routed: number of stage-2 rows fed by this (token, source) slot
   int dst[kDstRegs];  //                  and those rows (when K <= kDstRegs)
+  float wsc[kDstRegs];//                  weight of the path behind each destination (projection-side reuse only)
   bool dst_in_regs;
 };
 
-template <int STAGE>
+template <int STAGE, bool MERGE>
 __device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, const TileInfo &t, int r) {
   RowCtx c;
   const bool valid = r < t.valid;
@@ -157,9 +160,13 @@ __device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, c
     for (int k = 0; k < kDstRegs; ++k) {
       if (k < p.K && S.path_prow1[(size_t)c.token * p.K + k] == c.my_prow) {
         const int d = S.path_pos2[(size_t)c.token * p.K + k];
+        const float wk = MERGE ? S.path_w[(size_t)c.token * p.K + k] : 0.0f;
 #pragma unroll
         for (int j = 0; j < kDstRegs; ++j)
-          if (j == c.nd) c.dst[j] = d;
+          if (j == c.nd) {
+            c.dst[j] = d;
+            if (MERGE) c.wsc[j] = wk;
+          }
         ++c.nd;
       }
     }
@@ -180,15 +187,39 @@ __device__ __forceinline__ void swiglu_pack32(const uint32_t (&g)[32], const uin
   }
 }
 
+// Eight bf16 values scaled by `sc` and added to eight bf16 values in global memory (a stage-2 row that several
+// paths of a token feed: the row starts from zero and collects beta * U of each of them).
+__device__ __forceinline__ void red_add_scaled_bf16x8(__nv_bfloat16 *addr, uint4 x, float sc) {
+  uint32_t *w = reinterpret_cast<uint32_t *>(&x);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h2 = *reinterpret_cast<__nv_bfloat162 *>(&w[i]);
+    const float2 f = __bfloat1622float2(h2);
+    h2 = __floats2bfloat162_rn(f.x * sc, f.y * sc);
+    w[i] = *reinterpret_cast<uint32_t *>(&h2);
+  }
+  asm volatile("red.global.add.noftz.v4.bf16x2 [%0], {%1, %2, %3, %4};" ::"l"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3])
+               : "memory");
+}
+
 // Direct store of 32 bf16 of this thread's row to every path that reuses it, looked up on the spot
 // (only when a token has more paths than the destination registers hold).
+template <bool MERGE>
 __device__ __forceinline__ void store_row_lookup(const TcParams &p, const Seg &S, const RowCtx &c, size_t col,
                                                  const uint4 (&out)[4]) {
   for (int k = 0; k < p.K; ++k) {
     if (S.path_prow1[(size_t)c.token * p.K + k] != c.my_prow) continue;
-    uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)S.path_pos2[(size_t)c.token * p.K + k] * S.ldu + col);
+    const int d = S.path_pos2[(size_t)c.token * p.K + k];
+    if (d >= 0) {
+      uint4 *d4 = reinterpret_cast<uint4 *>(S.u_out + (size_t)d * S.ldu + col);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) d4[q] = out[q];
+      for (int q = 0; q < 4; ++q) d4[q] = out[q];
+    } else if (MERGE && d <= -2) {
+      const float sc = S.path_w[(size_t)c.token * p.K + k];
+      __nv_bfloat16 *dr = S.u_out + (size_t)(-d - 2) * S.ldu + col;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) red_add_scaled_bf16x8(dr + 8 * q, out[q], sc);
+    }
   }
 }
 
@@ -215,7 +246,7 @@ __device__ __forceinline__ void scatter_add_32x32(const TcParams &p, float *stag
 // Drains one accumulator (this thread's TMEM lane) and applies the stage's epilogue.  TMEM loads are issued
 // one step ahead of the arithmetic: a tcgen05.ld queues behind the MMAs already issued, so its latency is
 // long while the next tile is being computed, and must overlap the math and the stores of the previous step.
-template <int STAGE>
+template <int STAGE, bool MERGE>
 __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, const TileInfo &t, const RowCtx &c,
                                               uint32_t taddr, float *stage) {
   if (STAGE == 1) {
@@ -236,7 +267,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
       tmem_ld32_issue(taddr + c0 + 32, g1);
       tmem_ld32_issue(taddr + 128 + c0 + 32, u1);
       swiglu_pack32(g0, u0, out);
-      if (c.ok && !c.dst_in_regs) store_row_lookup(p, S, c, col0 + c0, out);
+      if (c.ok && !c.dst_in_regs) store_row_lookup<MERGE>(p, S, c, col0 + c0, out);
 #pragma unroll
       for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow)[q] = out[q];
       tmem_wait_ld();
@@ -246,22 +277,29 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
         tmem_ld32_issue(taddr + 128 + c0 + 64, u0);
       }
       swiglu_pack32(g1, u1, out);
-      if (c.ok && !c.dst_in_regs) store_row_lookup(p, S, c, col0 + c0 + 32, out);
+      if (c.ok && !c.dst_in_regs) store_row_lookup<MERGE>(p, S, c, col0 + c0 + 32, out);
 #pragma unroll
       for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow + 64)[q] = out[q];
       __syncwarp();
       for (int k = 0; k < max_nd; ++k) {
         int dk = -1;
+        float wk = 0.0f;
 #pragma unroll
         for (int j = 0; j < kDstRegs; ++j)
-          if (j == k && k < c.nd) dk = c.dst[j];
+          if (j == k && k < c.nd) {
+            dk = c.dst[j];
+            if (MERGE) wk = c.wsc[j];
+          }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int row = i * 4 + (lane >> 3);
           const int d = __shfl_sync(0xffffffffu, dk, row);
+          const float sc = MERGE ? __shfl_sync(0xffffffffu, wk, row) : 0.0f;
           const uint4 x = *reinterpret_cast<const uint4 *>(reinterpret_cast<unsigned char *>(stage) +
                                                            row * (kEpiStride * 4) + (lane & 7) * 16);
           if (d >= 0) *reinterpret_cast<uint4 *>(S.u_out + (size_t)d * S.ldu + col0 + c0 + (lane & 7) * 8) = x;
+          else if (MERGE && d <= -2)
+            red_add_scaled_bf16x8(S.u_out + (size_t)(-d - 2) * S.ldu + col0 + c0 + (lane & 7) * 8, x, sc);
         }
       }
       __syncwarp();
@@ -290,7 +328,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
 
 // STAGE = 1: SwiGLU epilogue (B = 128 gate rows | 128 up rows);  STAGE = 2: weighted scatter-add epilogue.
 // Tensor maps: A, B (gate or down), B2 (up; unused in stage 2) for segment 0 and for segment 1.
-template <int STAGE>
+template <int STAGE, bool MERGE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                     const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
@@ -432,10 +470,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       const TileInfo t = walk.at(tile);
       const Seg &S = p.seg[t.seg];
-      const RowCtx c = prepare_row<STAGE>(p, S, t, r);
+      const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
+      epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
                            s_epi + (warp - 2) * 32 * kEpiStride);
       tc_fence_before();
       mbar_arrive(acce_bar(acc));
@@ -553,7 +591,7 @@ struct PairWalker {
   }
 };
 
-template <int STAGE>
+template <int STAGE, bool MERGE = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                          const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
@@ -712,10 +750,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
     for (int tile = pair_id; tile < total; tile += n_pairs) {
       const TileInfo t = walk.at(tile, rank);
       const Seg &S = p.seg[t.seg];
-      const RowCtx c = prepare_row<STAGE>(p, S, t, r);
+      const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile<STAGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
+      epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
                            s_epi + (warp - 2) * 32 * kEpiStride);
       tc_fence_before();
       mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));   // the leader's MMA waits for both halves
@@ -742,8 +780,11 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
 // Copies rows idx[r] of src into consecutive rows of dst (the A operand of stage 1 in group order); a negative
 // index marks a padding row, which is written as zeros (zero operands keep the tensor cores' switching power
 // down for rows whose results are dropped).  One warp per row; up to eight 16-byte loads in flight per lane.
+// With projection-side reuse it also clears the stage-2 rows that several paths of a token feed (stored in the
+// path map as -(row + 2)), which stage 1 then fills by adding.
 __global__ void __launch_bounds__(256) gather_rows_kernel(uint4 *dst, const uint4 *src, const int32_t *idx,
-                                                          const int32_t *tile_base, int G, int vec_per_row) {
+                                                          const int32_t *tile_base, int G, int vec_per_row,
+                                                          const int32_t *pos2, int n_paths, uint4 *u, int u_vec_per_row) {
   pdl_grid_wait();
   const int rows = tile_base[G] * kTileM;
   const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
@@ -764,6 +805,14 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(uint4 *dst, const uint
         const int v = v0 + i * 32 + lane;
         if (v < vec_per_row) d[v] = x[i];
       }
+    }
+  }
+  if (pos2) {
+    for (int q = blockIdx.x * warps_per_block + (threadIdx.x >> 5); q < n_paths; q += gridDim.x * warps_per_block) {
+      const int d = pos2[q];
+      if (d > -2) continue;
+      uint4 *row = u + (size_t)(-d - 2) * u_vec_per_row;
+      for (int v = lane; v < u_vec_per_row; v += 32) row[v] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
 }
@@ -798,12 +847,15 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     attr_done = true;
   }
   // CTA pairs pay off once groups are a few tiles long; short groups (decode) leave the peer CTA idle
   const bool pair = c.ffn_impl == PCOMOE_FFN_TCGEN05_PAIR ||
                     (c.ffn_impl == PCOMOE_FFN_AUTO && (int64_t)T * c.top_k >= (int64_t)256 * n);
   const int grid = pair ? (L->sm_count & ~1) : L->sm_count;
+  const bool merge = c.target_reuse != 0;
   const uint32_t down_box = pair ? 128 : 256;   // a CTA of a pair loads half of the 256-row slice of W_down
 
   // ---- stage 1: rows of h gathered into group order, then one launch over routed + shared tiles ----
@@ -815,13 +867,16 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     bool ok = true;
     if (stages & kStage1Routed) {
       PCOMOE_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3(L->sm_count * 8), dim3(256), 0, st, Hg,
-                                 reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8));
+                                 reinterpret_cast<const uint4 *>(h), a1, tb1, n, H / 8,
+                                 merge ? pos2 : (const int32_t *)nullptr, (int)(T * c.top_k),
+                                 reinterpret_cast<uint4 *>(U), F / 8));
       count_launch();
       ok = ok && make_map(&mA[ns], Hg, pad_rows, H, kTileM) && make_map(&mB[ns], wg, (uint64_t)n * F, H, 128) &&
            make_map(&mC[ns], wu, (uint64_t)n * F, H, 128);
       Seg &S = p.seg[ns++];
       S.tile_base = tb1; S.row_offsets = g->s1_offsets; S.G = n; S.nt = F / 128; S.kb = H / BK; S.b_group_rows = F;
       S.row_token = a1; S.path_prow1 = prow1; S.path_pos2 = pos2; S.u_out = U; S.ldu = F;
+      S.path_w = merge ? reinterpret_cast<const float *>(ws + lay.path_wgt) : nullptr;
     }
     if (stages & kStage1Shared) {
       ok = ok && make_map(&mA[ns], h, (uint64_t)T, H, kTileM) && make_map(&mB[ns], sg, Fsh, H, 128) &&
@@ -836,8 +891,9 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
       p.zero_ptr = reinterpret_cast<float4 *>(y);
       p.zero_vec4 = (int64_t)T * H / 4;
     }
-    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<1> : grouped_gemm_kernel<1>, dim3(grid), dim3(kThreads),
-                               kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
+    auto k3 = merge ? (pair ? grouped_gemm_pair_kernel<1, true> : grouped_gemm_kernel<1, true>)
+                    : (pair ? grouped_gemm_pair_kernel<1, false> : grouped_gemm_kernel<1, false>);
+    PCOMOE_CUDA_TRY(launch_pdl(k3, dim3(grid), dim3(kThreads), kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
     count_launch();
   }
 

@@ -24,7 +24,9 @@ struct GroupParams {
   int32_t *blk_cnt;                   // [2][n][NB]: per-block counts, turned into per-block offsets by the scan
   int32_t *a1_idx;                    // token of every padded stage-1 row
   int32_t *path_prow1, *path_pos2;    // [T,K] padded stage-1 / stage-2 row of every path
+  float *path_wgt;                    // [T,K] copy of the path weights (projection-side reuse only)
   int32_t T, n, K, dedup, chunk, nb;
+  int32_t tgt_reuse;                  // 1: stage-2 rows are unique (token, target) pairs
 };
 
 __device__ __forceinline__ void flag_error(DevPlan *plan, int code) { atomicCAS(&plan->status, 0, code); }
@@ -67,7 +69,7 @@ __global__ void group_count_kernel(const GroupParams p) {
     for (int k = 0; k < p.K; ++k) {
       if (rs[k] < 0) continue;
       if (first_occurrence(rs, k, p.dedup) == k) atomicAdd(&h1[rs[k]], 1);
-      atomicAdd(&h2[rt[k]], 1);
+      if (first_occurrence(rt, k, p.tgt_reuse) == k) atomicAdd(&h2[rt[k]], 1);
     }
   }
   __syncthreads();
@@ -169,8 +171,8 @@ __device__ __forceinline__ int bits_below(const uint32_t *row, int idx) {
 __device__ __forceinline__ void scatter_block(const GroupParams &p, int32_t *sm, const int32_t *cnt, bool single) {
   const int CK = p.chunk * p.K;
   const int W = (CK + 31) >> 5;
-  int32_t *ssrc = sm, *stgt = ssrc + CK, *srow = stgt + CK;
-  int32_t *off1 = srow + CK, *off2 = off1 + p.n, *tb1 = off2 + p.n, *tb2 = tb1 + p.n;
+  int32_t *ssrc = sm, *stgt = ssrc + CK, *srow = stgt + CK, *spos = srow + CK;
+  int32_t *off1 = spos + CK, *off2 = off1 + p.n, *tb1 = off2 + p.n, *tb2 = tb1 + p.n;
   int32_t *bo1 = tb2 + p.n, *bo2 = bo1 + p.n;
   uint32_t *bits1 = reinterpret_cast<uint32_t *>(bo2 + p.n), *bits2 = bits1 + (size_t)p.n * W;
 
@@ -203,7 +205,7 @@ __device__ __forceinline__ void scatter_block(const GroupParams &p, int32_t *sm,
       if (rs[k] < 0) continue;
       const int idx = tl * p.K + k;
       if (first_occurrence(rs, k, p.dedup) == k) atomicOr(&bits1[(size_t)rs[k] * W + (idx >> 5)], 1u << (idx & 31));
-      atomicOr(&bits2[(size_t)rt[k] * W + (idx >> 5)], 1u << (idx & 31));
+      if (first_occurrence(rt, k, p.tgt_reuse) == k) atomicOr(&bits2[(size_t)rt[k] * W + (idx >> 5)], 1u << (idx & 31));
     }
   }
   __syncthreads();
@@ -233,16 +235,30 @@ __device__ __forceinline__ void scatter_block(const GroupParams &p, int32_t *sm,
       p.path_pos2[(size_t)t * p.K + k] = -1;
       continue;
     }
-    const int idx = tl * p.K + k;
-    const int r2 = off2[j] + bo2[j] + bits_below(bits2 + (size_t)j * W, idx);
     const int q = t * p.K + k;
     const int s = rs[k];
-    p.g.s2_path[r2] = q;
-    p.g.s2_s1row[r2] = myrow[k];
-    p.g.s2_token[r2] = t;
-    p.g.s2_w[r2] = p.w[q];
+    int32_t *mypos = spos + tl * p.K;
+    const int fk = first_occurrence(rt, k, p.tgt_reuse);
+    if (fk == k) {
+      // with projection-side reuse a row fed by several of the token's paths is marked: its position is stored
+      // as -(position + 2), its weight is 1, and stage 1 adds the weighted intermediates into it
+      bool merged = false;
+      if (p.tgt_reuse)
+        for (int k2 = k + 1; k2 < p.K; ++k2) merged |= rt[k2] == j;
+      const int idx = tl * p.K + k;
+      const int r2 = off2[j] + bo2[j] + bits_below(bits2 + (size_t)j * W, idx);
+      p.g.s2_path[r2] = q;
+      p.g.s2_s1row[r2] = myrow[k];
+      p.g.s2_token[r2] = t;
+      p.g.s2_w[r2] = merged ? 1.0f : p.w[q];
+      const int pos = tb2[j] * kTileM + (r2 - off2[j]);
+      mypos[k] = merged ? -(pos + 2) : pos;
+    } else {
+      mypos[k] = mypos[fk];
+    }
     p.path_prow1[q] = tb1[s] * kTileM + (myrow[k] - off1[s]);
-    p.path_pos2[q] = tb2[j] * kTileM + (r2 - off2[j]);
+    p.path_pos2[q] = mypos[k];
+    if (p.tgt_reuse) p.path_wgt[q] = p.w[q];
   }
 }
 
@@ -270,7 +286,7 @@ __global__ void group_single_block_kernel(const GroupParams p) {
       for (int k = 0; k < p.K; ++k) {
         if (rs[k] < 0) continue;
         if (first_occurrence(rs, k, p.dedup) == k) atomicAdd(&cnt[rs[k]], 1);
-        atomicAdd(&cnt[p.n + rt[k]], 1);
+        if (first_occurrence(rt, k, p.tgt_reuse) == k) atomicAdd(&cnt[p.n + rt[k]], 1);
       }
     }
     __syncthreads();
@@ -293,11 +309,13 @@ pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src
   p.path_prow1 = reinterpret_cast<int32_t *>(ws + lay.path_prow1);
   p.path_pos2 = reinterpret_cast<int32_t *>(ws + lay.path_pos2);
   p.T = T; p.n = c.n_experts; p.K = c.top_k; p.dedup = c.dedup; p.chunk = group_chunk_for(L, T);
+  p.tgt_reuse = c.target_reuse;
+  p.path_wgt = c.target_reuse ? reinterpret_cast<float *>(ws + lay.path_wgt) : nullptr;
   p.nb = (T + p.chunk - 1) / p.chunk;
 
   const int CK = p.chunk * p.K, W = (CK + 31) / 32;
   const size_t smem_count = sizeof(int32_t) * ((size_t)2 * CK + 2 * p.n);
-  const size_t smem_scatter = sizeof(int32_t) * ((size_t)3 * CK + 6 * p.n + (size_t)2 * p.n * W);
+  const size_t smem_scatter = sizeof(int32_t) * ((size_t)4 * CK + 6 * p.n + (size_t)2 * p.n * W);
   if (smem_scatter > 200 * 1024) return PCOMOE_ERR_UNSUPPORTED;
   if (smem_count > 48 * 1024)
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(group_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_count));

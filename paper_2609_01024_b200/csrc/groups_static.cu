@@ -50,6 +50,7 @@ extern "C" pcomoe_status pcomoe_build_path_groups_static(const pcomoe_layer *L, 
   if (T < 0) return PCOMOE_ERR_SHAPE;
   if (T > 0 && (!d_path_src || !d_path_tgt || !d_path_w)) return PCOMOE_ERR_INVALID_ARG;
   if ((int64_t)T * L->cfg.top_k >= (int64_t)1 << 31) return PCOMOE_ERR_SHAPE;
+  if (L->cfg.target_reuse) return PCOMOE_ERR_UNSUPPORTED;   // that mode keeps a per-path array beyond the scratch
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return PCOMOE_ERR_CUDA;
   if (dev != L->device) return PCOMOE_ERR_INVALID_ARG;   // the layer's table lives on its own device

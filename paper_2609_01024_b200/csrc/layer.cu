@@ -48,6 +48,7 @@ WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
   w.u = take(es * (size_t)w.mt_max * kTileM * c.ffn);
   w.u_sh = take(es * (size_t)w.t_pad * c.shared_ffn);
   if (L->tc_ok) w.h_gath = take(es * (size_t)w.mt_max * kTileM * c.hidden);
+  if (c.target_reuse) w.path_wgt = take(sizeof(float) * (size_t)Pm);
   w.total = off;
   return w;
 }
@@ -59,7 +60,14 @@ extern "C" {
 pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mask,
                                   const float *h_bias, pcomoe_layer **out) {
   if (!cfg || !h_mask || !h_bias || !out) return PCOMOE_ERR_INVALID_ARG;
-  if (cfg->struct_size != (int32_t)sizeof(pcomoe_config)) return PCOMOE_ERR_INVALID_ARG;
+  // the struct may end before `target_reuse` (the layout before that field was added)
+  const int32_t old_size = (int32_t)offsetof(pcomoe_config, target_reuse);
+  if (cfg->struct_size != (int32_t)sizeof(pcomoe_config) && cfg->struct_size != old_size) return PCOMOE_ERR_INVALID_ARG;
+  pcomoe_config full = {};
+  std::memcpy(&full, cfg, (size_t)cfg->struct_size);
+  full.struct_size = (int32_t)sizeof(pcomoe_config);
+  cfg = &full;
+  if (cfg->target_reuse != 0 && cfg->target_reuse != 1) return PCOMOE_ERR_INVALID_ARG;
   const int n = cfg->n_experts, K = cfg->top_k;
   if (n <= 0 || K <= 0 || cfg->hidden <= 0 || cfg->ffn <= 0 || cfg->shared_ffn < 0)
     return PCOMOE_ERR_INVALID_ARG;
@@ -79,6 +87,11 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
   L->tc_ok = cfg->in_dtype == PCOMOE_BF16 && cfg->hidden % 256 == 0 && cfg->ffn % 128 == 0 &&
              cfg->shared_ffn % 128 == 0;
   if (cfg->ffn_impl >= PCOMOE_FFN_TCGEN05 && !L->tc_ok) {
+    delete L;
+    return PCOMOE_ERR_UNSUPPORTED;
+  }
+  // projection-side reuse lives in the tensor-core epilogue only
+  if (cfg->target_reuse && (!L->tc_ok || cfg->ffn_impl == PCOMOE_FFN_SIMT)) {
     delete L;
     return PCOMOE_ERR_UNSUPPORTED;
   }
@@ -105,7 +118,7 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
   int chunk = 128;
   auto scatter_smem = [&](int ch) {
     const size_t ck = (size_t)ch * K, words = (ck + 31) / 32;
-    return 4 * (3 * ck + 6 * (size_t)n + 2 * (size_t)n * words);
+    return 4 * (4 * ck + 6 * (size_t)n + 2 * (size_t)n * words);
   };
   while (chunk > 32 && scatter_smem(chunk) > 96 * 1024) chunk >>= 1;
   L->group_chunk = chunk;
