@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol(lib):
 def test_binding_lists_the_same_symbols():
     from paper_2609_01024_b200 import binding
     assert sorted(binding.EXPORTS) == _declared()
-    assert ctypes.sizeof(binding.pcomoe_config) == 13 * 4
+    assert ctypes.sizeof(binding.pcomoe_config) == 14 * 4
 
 
 def test_host_side_argument_checks(lib):
@@ -57,5 +57,19 @@ def test_host_side_argument_checks(lib):
     cfg.hidden = 64
     cfg.ffn_impl = 2                                                                             # tcgen05 needs H % 256
     assert lib.pcomoe_layer_create(ctypes.byref(cfg), mask, bias, ctypes.byref(out)) == 4
+    cfg.ffn_impl = 0
+    cfg.target_reuse = 1                                                                         # needs the tensor-core path
+    assert lib.pcomoe_layer_create(ctypes.byref(cfg), mask, bias, ctypes.byref(out)) == 4
+    cfg.target_reuse = 7
+    assert lib.pcomoe_layer_create(ctypes.byref(cfg), mask, bias, ctypes.byref(out)) == 1
+    cfg.target_reuse = 0
+    cfg.struct_size = 12                                                                         # neither layout
+    assert lib.pcomoe_layer_create(ctypes.byref(cfg), mask, bias, ctypes.byref(out)) == 1
     assert lib.pcomoe_route_paths(None, 4, None, None, None, None, None, None) == 1
+    assert lib.pcomoe_router_logits(None, 4, None, None, None, None, 0, ctypes.c_float(1.0), None, None, 0, None) == 1
+    assert lib.pcomoe_residual_cast(None, 4, None, None, None, None) == 1
+    assert lib.pcomoe_mask_tighten(4, None, None, ctypes.c_float(0.5), None) == 1
+    m2 = (ctypes.c_uint8 * 16)(*([1] * 16))
+    assert lib.pcomoe_mask_tighten(4, bias, m2, ctypes.c_float(0.5), m2) == 0                    # in place
+    assert sum(m2) == 4 + 6
     assert lib.pcomoe_device_status(None, None) == 3
