@@ -199,6 +199,38 @@ def run_reference(args, cfg):
     print(json.dumps(out), flush=True)
 
 
+def density_sweep(args, cfg, L, layer0, d_logits, d_h, dev, stream):
+    """Time of one step and reuse statistics against the density of the compatibility mask (Sec. 5.3 reports path
+    density and reuse savings per block of the trained models; here the mask is the recipe's, thresholded at p)."""
+    import torch
+    from paper_2609_01024_b200 import binding as B
+    dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
+    rows = []
+    for p_on in (0.0, 0.1, 0.25, 0.5, 0.75, 1.0):
+        mask = wl.make_mask(cfg.scaled(mask_p=p_on))
+        lay = B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=cfg.F, mask=mask, bias=L.bias,
+                             w_gate=layer0.w_gate, w_up=layer0.w_up, w_down=layer0.w_down,
+                             shared=layer0.shared if cfg.F_sh else None, max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam,
+                             ffn_impl=args.ffn_impl, target_reuse=args.target_reuse, device=dev)
+        torch.cuda.synchronize()
+        time.sleep(1.0)      # every point starts from the same idle power state as the headline measurement
+        for _ in range(args.warmup):
+            lay.forward(d_logits, d_h)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.steps):
+            lay.forward(d_logits, d_h)
+        b.record(stream)
+        torch.cuda.synchronize()
+        st = lay.groups.stats.cpu().numpy()
+        P = cfg.T * cfg.K
+        rows.append({"mask_p": p_on, "active_paths": int(mask.sum()), "ms_per_step": a.elapsed_time(b) / args.steps,
+                     "R1_over_P": int(st[0]) / P, "stage2_rows_over_P": int(st[1]) / P,
+                     "expert_flops_saved": 1.0 - (2 * int(st[0]) + int(st[1])) / (3.0 * P)})
+        del lay
+    return rows
+
+
 def run_stack(args, cfg, L, layer0, d_h, dev, rank, world, stream):
     """Decode step through `--layers` blocks.  Every block has its own mask, bias and router (seeded per block; the
     first two keep every path, Sec. 5.3) and its own copy of the expert weights in HBM, so that every step streams
@@ -305,6 +337,9 @@ def main():
                          "0 = none, in front of the path gate); default -1: logits are an input, as the metric is quoted")
     ap.add_argument("--target-reuse", type=int, default=0,
                     help="1: projection-side reuse (one stage-2 row per unique (token, target), exact by linearity)")
+    ap.add_argument("--sweep-density", action="store_true",
+                    help="also time the layer at mask densities 0 (diagonal only) .. 1 (every path) and add the list "
+                         "as \"density_sweep\" to the JSON line (nested masks: the recipe's uniforms thresholded at p)")
     ap.add_argument("--layers", type=int, default=0,
                     help="L > 0: time a decode step through a stack of L blocks (router + path gate + FFN + residual "
                          "per block, one CUDA graph per step) instead of the single-layer metric")
@@ -492,6 +527,8 @@ def main():
                                   "frac_of_measured": t_roof_meas / (ms_per_step * 1e-3),
                                   "frac_of_nominal_2.25PF_8TBs": t_roof_nominal / (ms_per_step * 1e-3)},
                "stage_ms": stage_ms}
+        if args.sweep_density and world == 1:
+            out["density_sweep"] = density_sweep(args, cfg, L, layer, d_logits, d_h, dev, stream)
         if not args.no_cpu_baseline and world == 1:
             n_cpu = args.cpu_tokens
             if n_cpu <= 0:   # probe with a few tokens per thread, then size the sample for about 20 s
