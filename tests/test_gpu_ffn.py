@@ -160,3 +160,23 @@ def test_cuda_graph_replay_matches_eager(G, oracle):
     rs, rt, rw = oracle.route(z2, L.mask, L.bias, cfg.lam, cfg.K)
     assert np.array_equal(layer.path_src[:cfg.T].cpu().numpy(), rs)
     G.check_output(y, oracle.ffn(wl.hidden_as_f32(cfg2, h2), L.w_gate, L.w_up, L.w_down, rs, rt, rw))
+
+
+@pytest.mark.parametrize("impl", [2, 3])
+def test_every_token_on_one_source(G, oracle, impl):
+    """Degenerate load: one expert's logit dominates, so every path of every token has the same source - a single
+    stage-1 group of T rows (several tiles and a ragged tail), all other source groups empty."""
+    import torch
+    cfg = wl.small_case(91, T=700, H=256, F=256, n=8, K=2, mask_p=1.0)
+    L = wl.make_layer(cfg)
+    z = L.logits.copy()
+    z[:, 3] += 100.0
+    layer = G.make_gpu_layer(cfg, L, ffn_impl=impl)
+    y = layer.forward(torch.from_numpy(z).to(layer.device), G.B.to_device(L.h)).cpu().numpy()
+    assert layer.device_status() == 0
+    rs, rt, rw = oracle.route(z, L.mask, L.bias, cfg.lam, cfg.K)
+    assert np.all(rs == 3)
+    assert np.array_equal(layer.path_src[:cfg.T].cpu().numpy(), rs) and np.array_equal(layer.path_tgt[:cfg.T].cpu().numpy(), rt)
+    g = layer.groups.to_host()
+    assert g["R1"] == cfg.T and int(g["stats"][4]) == cfg.n - 1
+    G.check_output(y, oracle.ffn(wl.hidden_as_f32(cfg, L.h), L.w_gate, L.w_up, L.w_down, rs, rt, rw))
