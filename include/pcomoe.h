@@ -245,6 +245,21 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, co
                                         const pcomoe_groups *groups, void *d_y, void *d_workspace,
                                         size_t ws_bytes, void *stream, int32_t stages);
 
+/* The whole hot path in one call: pcomoe_route_paths, pcomoe_build_path_groups and pcomoe_ffn_forward with the
+ * same arguments and the same results.  What the single call adds: on prefill-sized batches of a tensor-core
+ * layer with a shared expert, the shared expert's stage 1 (which depends on none of the routing) runs on a second
+ * stream that the layer owns, beside the routing, grouping and row-gather kernels, and is joined before stage 2.
+ * The second stream is ordered against `stream` with events on both sides, so the call behaves like work on
+ * `stream` alone and can be recorded into a CUDA graph.  One call per layer at a time.  A wait that ran out in the
+ * side launch is reported through the router's status word (see pcomoe_device_status).
+ * Arguments as in the three calls (d_path_* and the arrays of `groups` are outputs).  Errors: theirs. */
+pcomoe_status pcomoe_layer_forward(const pcomoe_layer *layer, int32_t T, const float *d_logits,
+                                   const float *d_tgt_logits, const void *d_h, const void *d_w_gate,
+                                   const void *d_w_up, const void *d_w_down, const void *d_wsh_gate,
+                                   const void *d_wsh_up, const void *d_wsh_down, int32_t *d_path_src,
+                                   int32_t *d_path_tgt, float *d_path_w, const pcomoe_groups *groups, void *d_y,
+                                   void *d_workspace, size_t ws_bytes, void *stream);
+
 /* Router in front of the path gate (Sec. 3.1: the router maps a token's hidden state to routing scores;
  * Sec. 4.2 uses them as the base routing signal g_base(h), and as g_tgt(h) unless a second head is given):
  *     d_logits[t,e] = sum_k d_h[t,k] * d_w_router[e,k]

@@ -22,7 +22,7 @@ PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR = 
 
 EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_mask_tighten", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
            "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",
-           "pcomoe_ffn_forward_stages", "pcomoe_router_logits", "pcomoe_residual_cast",
+           "pcomoe_ffn_forward_stages", "pcomoe_layer_forward", "pcomoe_router_logits", "pcomoe_residual_cast",
            "pcomoe_device_status",
            "pcomoe_launch_count", "pcomoe_status_string"]
 
@@ -70,6 +70,7 @@ def load_library(path: str | None = None):
     lib.pcomoe_build_path_groups_static.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp]
     lib.pcomoe_ffn_forward.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
     lib.pcomoe_ffn_forward_stages.argtypes = lib.pcomoe_ffn_forward.argtypes + [i32]
+    lib.pcomoe_layer_forward.argtypes = [vp, i32] + [vp] * 12 + [ctypes.POINTER(pcomoe_groups), vp, vp, sz, vp]
     lib.pcomoe_router_logits.argtypes = [vp, i32, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, sz, vp]
     lib.pcomoe_residual_cast.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.pcomoe_device_status.argtypes = [vp, vp]
@@ -223,6 +224,15 @@ def pcomoe_ffn_forward_stages(layer, T, h, w_gate, w_up, w_down, wsh_gate, wsh_u
                                                     stages), "pcomoe_ffn_forward_stages")
 
 
+def pcomoe_layer_forward(layer, T, logits, tgt_logits, h, w_gate, w_up, w_down, wsh_gate, wsh_up, wsh_down, path_src,
+                         path_tgt, path_w, groups: Groups, y, workspace):
+    _check(load_library().pcomoe_layer_forward(layer, T, _ptr(logits), _ptr(tgt_logits), _ptr(h), _ptr(w_gate), _ptr(w_up),
+                                               _ptr(w_down), _ptr(wsh_gate), _ptr(wsh_up), _ptr(wsh_down),
+                                               _ptr(path_src), _ptr(path_tgt), _ptr(path_w), ctypes.byref(groups.c),
+                                               _ptr(y), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                               _stream()), "pcomoe_layer_forward")
+
+
 def pcomoe_router_logits(layer, T, h, w_router, lora_a, lora_b, lora_rank: int, lora_scale: float, logits, workspace):
     _check(load_library().pcomoe_router_logits(layer, T, _ptr(h), _ptr(w_router), _ptr(lora_a), _ptr(lora_b),
                                                lora_rank, lora_scale, _ptr(logits), _ptr(workspace),
@@ -320,6 +330,14 @@ class PathMoELayer:
 
     def forward(self, logits, h, tgt_logits=None):
         """The whole hot path on device tensors: route -> group -> stage 1 -> stage 2.  Returns y [T,H] fp32."""
+        T = h.shape[0]
+        assert T <= self.max_tokens
+        pcomoe_layer_forward(self.layer, T, logits, tgt_logits, h, self.w_gate, self.w_up, self.w_down, *self.shared,
+                             self.path_src, self.path_tgt, self.path_w, self.groups, self.y, self.workspace)
+        return self.y[:T]
+
+    def forward_three_calls(self, logits, h, tgt_logits=None):
+        """The same through the three separate entry points (route, group, FFN), everything on one stream."""
         T = h.shape[0]
         assert T <= self.max_tokens
         self.route(logits, tgt_logits)

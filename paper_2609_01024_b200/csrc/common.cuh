@@ -66,6 +66,8 @@ struct pcomoe_layer {
   int sm_count;
   int group_chunk;                  // tokens per block of the grouping kernels
   int tc_ok;                        // sizes and dtype allow the tcgen05 path
+  cudaStream_t side_stream;         // pcomoe_layer_forward: the shared expert's stage 1 runs here beside the routing chain
+  cudaEvent_t ev_fork, ev_join;     //                       ordering of side_stream against the caller's stream
 };
 
 namespace pcomoe {
@@ -77,6 +79,13 @@ inline size_t dtype_size(int dt) { return dt == PCOMOE_BF16 ? 2 : 4; }
 
 // Tokens per block of the grouping kernels for a batch of T tokens: the largest chunk the layer allows
 // (shared-memory bound), halved while that would leave fewer than two blocks per SM.
+// CTA pairs pay off once groups are a few tiles long; short groups (decode) leave the peer CTA idle
+inline bool use_cta_pairs(const pcomoe_layer *L, int32_t T) {
+  const pcomoe_config &c = L->cfg;
+  return c.ffn_impl == PCOMOE_FFN_TCGEN05_PAIR ||
+         (c.ffn_impl == PCOMOE_FFN_AUTO && (int64_t)T * c.top_k >= (int64_t)256 * c.n_experts);
+}
+
 inline int group_chunk_for(const pcomoe_layer *L, int32_t T) {
   int chunk = L->group_chunk;
   if (T <= chunk) return chunk;   // the whole batch fits one block
@@ -132,10 +141,13 @@ pcomoe_status launch_ffn_simt(const pcomoe_layer *L, int32_t T, const void *h, c
                               const void *wu, const void *wd, const void *sg, const void *su,
                               const void *sd, const pcomoe_groups *g, float *y, char *ws,
                               const WsLayout &lay, cudaStream_t st, int stages);
+pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const void *h, const void *sg,
+                                        const void *su, char *ws, const WsLayout &lay, cudaStream_t st);
 pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                             const void *wu, const void *wd, const void *sg, const void *su,
                             const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                            const WsLayout &lay, cudaStream_t st, int stages);
+                            const WsLayout &lay, cudaStream_t st, int stages,
+                            cudaEvent_t wait_before_stage2 = nullptr);
 
 // bits of `stages`
 constexpr int kStage1Routed = 1, kStage1Shared = 2, kStage2Routed = 4, kStage2Shared = 8;

@@ -591,7 +591,7 @@ struct PairWalker {
   }
 };
 
-template <int STAGE, bool MERGE = false>
+template <int STAGE, bool MERGE = false, int NST = STAGES2>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                          const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
@@ -600,7 +600,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   extern __shared__ unsigned char smem_dyn[];
   pdl_grid_wait();
   __shared__ int32_t s_tb[2 * (kMaxExperts + 2)], s_ro[2 * (kMaxExperts + 2)], s_pb[2 * (kMaxExperts + 2)];
-  __shared__ __align__(8) uint64_t s_bar[2 * STAGES2 + 4];
+  __shared__ __align__(8) uint64_t s_bar[2 * NST + 4];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ __align__(16) float s_epi[4 * 32 * kEpiStride];   // per epilogue warp: 32 rows being turned around
@@ -611,9 +611,9 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const uint32_t bar0 = smem_u32(s_bar);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES2 + s); };
-  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + a); };
-  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + 2 + a); };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (NST + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * NST + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * NST + 2 + a); };
 
   for (int sg = 0; sg < p.nseg; ++sg) {
     const Seg &S = p.seg[sg];
@@ -630,7 +630,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   }
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int s = 0; s < STAGES2; ++s) {
+    for (int s = 0; s < NST; ++s) {
       mbar_init(full_bar(s), 1);      // the leader's expect_tx arrival; bytes come from both CTAs
       mbar_init(empty_bar(s), 1);     // one commit (broadcast to both CTAs)
     }
@@ -700,7 +700,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
           tma_load_2d_pair(sa, mA, kb * BK, a_row, lead_full);
           tma_load_2d_pair(sb, mB, kb * BK, b_row, lead_full);
-          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+          if (++stage == NST) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -726,7 +726,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
           for (int k = 0; k < BK / 16; ++k)
             umma_bf16_pair(d_tmem, da + 2u * k, db + 2u * k, (kb | k) != 0 ? 1u : 0u);
           umma_commit_pair(empty_bar(stage));
-          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+          if (++stage == NST) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
         umma_commit_pair(accf_bar(acc));
@@ -822,10 +822,46 @@ static_assert((size_t)STAGES2 * STAGE2_BYTES + 1024 == kSmemDyn, "both kernels u
 
 }  // namespace
 
+// Stage 1 of the shared expert alone, with a 4-stage ring and the largest shared-memory carve-out, so that the
+// routing, grouping and gather kernels running on another stream at the same time fit on the same SMs (the
+// shared expert needs nothing from them).  Device-side problems go to the router's status word: the grouping
+// step running beside this launch clears the layer's own word.
+constexpr int kSideStages = 4;
+constexpr size_t kSmemSide = (size_t)kSideStages * STAGE2_BYTES + 1024;
+
+pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const void *h, const void *sg,
+                                        const void *su, char *ws, const WsLayout &lay, cudaStream_t st) {
+  const pcomoe_config &c = L->cfg;
+  const int H = c.hidden, Fsh = c.shared_ffn;
+  if (!L->tc_ok || Fsh <= 0) return PCOMOE_ERR_UNSUPPORTED;
+  DevPlan *plan = reinterpret_cast<DevPlan *>(ws + lay.plan);
+  __nv_bfloat16 *Ush = reinterpret_cast<__nv_bfloat16 *>(ws + lay.u_sh);
+  static bool attr_done = false;
+  auto kern = grouped_gemm_pair_kernel<1, false, kSideStages>;
+  if (!attr_done) {
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemSide));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+    attr_done = true;
+  }
+  CUtensorMap mA, mB, mC;
+  if (!(make_map(&mA, h, (uint64_t)T, H, kTileM) && make_map(&mB, sg, Fsh, H, 128) && make_map(&mC, su, Fsh, H, 128)))
+    return PCOMOE_ERR_CUDA;
+  TcParams p{};
+  p.K = c.top_k; p.T = T; p.y = nullptr; p.ldy = H;
+  // only the status word of the plan is touched by the kernel: point it at the router's word
+  p.plan = reinterpret_cast<DevPlan *>(reinterpret_cast<char *>(plan) + offsetof(DevPlan, status_router));
+  Seg &S = p.seg[0];
+  S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
+  p.nseg = 1;
+  PCOMOE_CUDA_TRY(launch_pdl(kern, dim3(L->sm_count & ~1), dim3(kThreads), kSmemSide, st, mA, mB, mC, mA, mB, mC, p));
+  count_launch();
+  return PCOMOE_OK;
+}
+
 pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                             const void *wu, const void *wd, const void *sg, const void *su,
                             const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                            const WsLayout &lay, cudaStream_t st, int stages) {
+                            const WsLayout &lay, cudaStream_t st, int stages, cudaEvent_t wait_before_stage2) {
   const pcomoe_config &c = L->cfg;
   if (!L->tc_ok) return PCOMOE_ERR_UNSUPPORTED;
   const int n = c.n_experts, H = c.hidden, F = c.ffn, Fsh = c.shared_ffn;
@@ -851,9 +887,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     attr_done = true;
   }
-  // CTA pairs pay off once groups are a few tiles long; short groups (decode) leave the peer CTA idle
-  const bool pair = c.ffn_impl == PCOMOE_FFN_TCGEN05_PAIR ||
-                    (c.ffn_impl == PCOMOE_FFN_AUTO && (int64_t)T * c.top_k >= (int64_t)256 * n);
+  const bool pair = use_cta_pairs(L, T);
   const int grid = pair ? (L->sm_count & ~1) : L->sm_count;
   const bool merge = c.target_reuse != 0;
   const uint32_t down_box = pair ? 128 : 256;   // a CTA of a pair loads half of the 256-row slice of W_down
@@ -898,6 +932,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   }
 
   // ---- stage 2: one launch over routed + shared tiles, accumulating into y ----
+  if (wait_before_stage2) PCOMOE_CUDA_TRY(cudaStreamWaitEvent(st, wait_before_stage2, 0));
   if (stages & (kStage2Routed | kStage2Shared)) {
     CUtensorMap mA[2], mB[2];
     TcParams p{};

@@ -126,10 +126,16 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
   cudaError_t e = cudaGetDevice(&L->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, L->device);
   if (e == cudaSuccess) e = cudaMalloc((void **)&L->d_table, sizeof(ActiveEntry) * (size_t)cnt);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess)
     e = cudaMemcpy(L->d_table, L->h_table, sizeof(ActiveEntry) * (size_t)cnt, cudaMemcpyHostToDevice);
   if (e != cudaSuccess) {
     if (L->d_table) cudaFree(L->d_table);
+    if (L->side_stream) cudaStreamDestroy(L->side_stream);
+    if (L->ev_fork) cudaEventDestroy(L->ev_fork);
+    if (L->ev_join) cudaEventDestroy(L->ev_join);
     std::free(L->h_table);
     delete L;
     return PCOMOE_ERR_CUDA;
@@ -174,6 +180,9 @@ pcomoe_status pcomoe_mask_tighten(int32_t n, const float *h_bias, const uint8_t 
 pcomoe_status pcomoe_layer_destroy(pcomoe_layer *L) {
   if (!L) return PCOMOE_ERR_INVALID_ARG;
   if (L->d_table) cudaFree(L->d_table);
+  if (L->side_stream) cudaStreamDestroy(L->side_stream);
+  if (L->ev_fork) cudaEventDestroy(L->ev_fork);
+  if (L->ev_join) cudaEventDestroy(L->ev_join);
   std::free(L->h_table);
   delete L;
   return PCOMOE_OK;
@@ -268,6 +277,54 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *L, int32_t T, const 
                          groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
   return launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
                          groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
+}
+
+pcomoe_status pcomoe_layer_forward(const pcomoe_layer *L, int32_t T, const float *d_logits,
+                                   const float *d_tgt_logits, const void *d_h, const void *d_w_gate,
+                                   const void *d_w_up, const void *d_w_down, const void *d_wsh_gate,
+                                   const void *d_wsh_up, const void *d_wsh_down, int32_t *d_path_src,
+                                   int32_t *d_path_tgt, float *d_path_w, const pcomoe_groups *groups, void *d_y,
+                                   void *d_workspace, size_t ws_bytes, void *stream) {
+  if (!L || !groups_ok(groups)) return PCOMOE_ERR_INVALID_ARG;
+  if (T < 0) return PCOMOE_ERR_SHAPE;
+  if (T == 0) return PCOMOE_OK;
+  if (!d_logits || !d_h || !d_w_gate || !d_w_up || !d_w_down || !d_path_src || !d_path_tgt || !d_path_w || !d_y)
+    return PCOMOE_ERR_INVALID_ARG;
+  if (L->cfg.shared_ffn > 0 && (!d_wsh_gate || !d_wsh_up || !d_wsh_down)) return PCOMOE_ERR_INVALID_ARG;
+  WsLayout lay;
+  pcomoe_status s = check_ws(L, T, d_workspace, ws_bytes, &lay);
+  if (s != PCOMOE_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool tc = L->cfg.ffn_impl >= PCOMOE_FFN_TCGEN05 || (L->cfg.ffn_impl == PCOMOE_FFN_AUTO && L->tc_ok);
+  // The shared expert's stage 1 needs nothing from routing, grouping and the row gather: on prefill-sized
+  // batches it runs on the layer's second stream beside them and joins before stage 2.
+  const bool overlap = tc && L->cfg.shared_ffn > 0 && use_cta_pairs(L, T);
+  if (overlap) {
+    PCOMOE_CUDA_TRY(cudaEventRecord(L->ev_fork, st));
+    PCOMOE_CUDA_TRY(cudaStreamWaitEvent(L->side_stream, L->ev_fork, 0));
+    s = launch_shared_stage1_side(L, T, d_h, d_wsh_gate, d_wsh_up, (char *)d_workspace, lay, L->side_stream);
+    // the join is recorded whatever happened, so that a stream capture always closes
+    PCOMOE_CUDA_TRY(cudaEventRecord(L->ev_join, L->side_stream));
+    if (s != PCOMOE_OK) {
+      cudaStreamWaitEvent(st, L->ev_join, 0);
+      return s;
+    }
+  }
+  s = launch_route(L, T, d_logits, d_tgt_logits ? d_tgt_logits : d_logits, d_path_src, d_path_tgt, d_path_w, st);
+  if (s == PCOMOE_OK)
+    s = launch_groups(L, T, d_path_src, d_path_tgt, d_path_w, groups, (char *)d_workspace, lay, st);
+  if (s == PCOMOE_OK) {
+    if (tc)
+      s = launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down, groups,
+                        (float *)d_y, (char *)d_workspace, lay, st,
+                        overlap ? (kStage1Routed | kStage2Routed | kStage2Shared) : 15, overlap ? L->ev_join : nullptr);
+    else
+      s = launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down, groups,
+                          (float *)d_y, (char *)d_workspace, lay, st, 15);
+  } else if (overlap) {
+    cudaStreamWaitEvent(st, L->ev_join, 0);
+  }
+  return s;
 }
 
 pcomoe_status pcomoe_router_logits(const pcomoe_layer *L, int32_t T, const void *d_h, const void *d_w_router,

@@ -180,3 +180,33 @@ def test_every_token_on_one_source(G, oracle, impl):
     g = layer.groups.to_host()
     assert g["R1"] == cfg.T and int(g["stats"][4]) == cfg.n - 1
     G.check_output(y, oracle.ffn(wl.hidden_as_f32(cfg, L.h), L.w_gate, L.w_up, L.w_down, rs, rt, rw))
+
+
+def test_single_call_forward_with_side_stream_matches_three_calls(G, oracle):
+    """pcomoe_layer_forward runs the shared expert's stage 1 on the layer's second stream; results are those of the
+    three separate calls, eagerly and when the call is recorded into a CUDA graph (the capture spans both streams)."""
+    import torch
+    cfg = wl.small_case(53, T=900, H=256, F=256, n=4, K=3, F_sh=512, mask_p=0.8)      # pairs + shared expert
+    L = wl.make_layer(cfg)
+    layer = G.make_gpu_layer(cfg, L)
+    dl, dh = torch.from_numpy(L.logits).to(layer.device), G.B.to_device(L.h)
+    y3 = layer.forward_three_calls(dl, dh).clone()
+    g3 = layer.groups.to_host()
+    y1 = layer.forward(dl, dh).clone()
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    g1 = layer.groups.to_host()
+    for k in G.GROUP_KEYS:
+        assert np.array_equal(np.asarray(g1[k]), np.asarray(g3[k])), k
+    rs, rt, rw = oracle.route(L.logits, L.mask, L.bias, cfg.lam, cfg.K)
+    yr = oracle.ffn(wl.hidden_as_f32(cfg, L.h), L.w_gate, L.w_up, L.w_down, rs, rt, rw,
+                    shared=(L.wsh_gate, L.wsh_up, L.wsh_down))
+    G.check_output(y1.cpu().numpy(), yr)
+    G.check_output(y3.cpu().numpy(), yr)
+    graph = layer.capture(dl, dh)
+    for _ in range(3):
+        layer.y.zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    G.check_output(layer.y[:cfg.T].cpu().numpy(), yr)
