@@ -85,7 +85,8 @@ typedef struct pcomoe_layer pcomoe_layer; /* opaque; owns the small device table
  * Layer set-up (offline, once per layer).  Builds the active set A = {(i,j) | m_ij = 1}
  * (Sec. 4.3, "Compositional Path Routing": path indices are materialised offline) as a compact
  * table sorted by flat id i*n+j, and copies it to the current device (the one call here that
- * allocates device memory; pcomoe_layer_destroy frees it).
+ * allocates device memory; it also creates the second stream and the two events that
+ * pcomoe_layer_forward uses; pcomoe_layer_destroy releases all of it).
  *   h_mask [n*n] uint8, row i = source, column j = target; every m_ii must be 1 (Sec. 4.2).
  *   h_bias [n*n] fp32 compatibility bias B; entries where the mask is 0 are never read.
  * Errors: INVALID_ARG (NULL, sizes <= 0, diagonal entry off), SHAPE (K > n or K > 32),
