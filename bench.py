@@ -64,6 +64,8 @@ class ClockSampler:
         self._stop = threading.Event()
 
     def start(self):
+        # both sources run: NVML answers every few milliseconds but its clock reading can lag a short timed region;
+        # nvidia-smi reports less often but reads the clocks itself
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -76,14 +78,16 @@ class ClockSampler:
             self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
             self.thread = threading.Thread(target=self._poll, daemon=True)
             self.thread.start()
-            return
         except Exception:
             self.nvml = None
         try:
+            sel = str(self.uuid) if self.uuid is not None else str(self.idx)
+            if self.uuid is not None and not sel.startswith("GPU-"):
+                sel = "GPU-" + sel
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.idx), "-lms", "100"], stdout=subprocess.PIPE, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
+                                          "-i", sel, "-lms", "20"], stdout=subprocess.PIPE, text=True)
+            self.thread2 = threading.Thread(target=self._read, daemon=True)
+            self.thread2.start()
         except Exception:
             self.proc = None
 
@@ -124,19 +128,17 @@ class ClockSampler:
         if self.nvml is not None:
             self._stop.set()
             self.thread.join(timeout=1.0)
-            pad0, pad1 = 0.0, 0.0
-        else:
-            time.sleep(0.15)
+        if self.proc is not None:
+            time.sleep(0.05)
             self.proc.terminate()
-            pad0, pad1 = 0.05, 0.15
         sm, mx, reasons = [], [], set()
-        for ts, mhz, mmax, rs in self.rows:
-            if t0 is not None and not (t0 - pad0 <= ts <= t1 + pad1):
+        for ts, mhz, mmax, rs in list(self.rows):
+            if t0 is not None and not (t0 <= ts <= t1 + 0.03):
                 continue
             sm.append(mhz); mx.append(mmax); reasons |= rs
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm),
-                "source": "nvml" if self.nvml is not None else "nvidia-smi"}
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm),
+                "source": "+".join(x for x, on in (("nvml", self.nvml is not None), ("nvidia-smi", self.proc is not None)) if on)}
 
 
 def algorithmic_work(cfg, R1, n_src, n_tgt):
