@@ -17,6 +17,12 @@
  * closed form; K=1; brute force over the dense n x n path grid; invariants.
  * The outputs y on the five benchmark layers have no printed value in the
  * paper: there the parity is pinned only through that chain.
+ * Router logits: a hand-computed case, unit-row weights, a library matrix product and
+ * the folded-weight identity.  Residual hand-over: hand cases around a bf16 rounding
+ * tie and an independent conversion.  Mask from bias / tightening step: closed cases,
+ * a numpy sort, nestedness along a schedule.  Target grouping with projection-side
+ * reuse: a hand example, sorted keys, the one-sixth count of Sec. 3.2 and a numpy
+ * evaluation of the layer over the merged rows.
  *
  * No blocking, fusion or reordering beyond what each equation states; OpenMP
  * is used only across tokens, which are independent.
