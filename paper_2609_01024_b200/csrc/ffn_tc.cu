@@ -42,6 +42,9 @@ struct Seg {
   int32_t nt;                  // tiles along N
   int32_t kb;                  // k-blocks
   int32_t b_group_rows;        // rows of the weight tensor per group (0 for a single group)
+  int32_t m_outer;             // tile order inside a group: 0 = the m-tiles of one n-tile run fastest (the group's rows
+                               // stay in L2 and its weights stream), 1 = the n-tiles of one m-tile run fastest (for a
+                               // group whose rows outweigh its weights: the shared expert on a large batch)
   // stage 1: where a row's SwiGLU output goes
   const int32_t *row_token;    // token of a padded row (routed), NULL: the row is its own destination
   const int32_t *path_prow1;   // [T,K] padded stage-1 row of every path
@@ -89,7 +92,7 @@ struct TileInfo {
 // that CTAs working at the same time share one slice of the group's weights.
 struct TileWalker {
   const int32_t *tb, *ro;      // [2][kMaxExperts + 2] each
-  int nt[2], G[2], nseg;
+  int nt[2], G[2], mo[2], nseg;
   int seg, g, seg_first;       // current segment, group, and the first tile id of the segment
   __device__ int seg_tiles(int s) const { return tb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
   __device__ int total() const {
@@ -111,8 +114,13 @@ struct TileWalker {
     const int local = local_seg - b[g] * n_t;
     t.seg = seg;
     t.g = g;
-    t.n_idx = local / mt;
-    t.m_idx = local - t.n_idx * mt;
+    if (mo[seg]) {
+      t.m_idx = local / n_t;
+      t.n_idx = local - t.m_idx * n_t;
+    } else {
+      t.n_idx = local / mt;
+      t.m_idx = local - t.n_idx * mt;
+    }
     t.prow0 = (b[g] + t.m_idx) * kTileM;
     t.urow0 = r[g] + t.m_idx * kTileM;
     t.valid = min(kTileM, r[g + 1] - t.urow0);
@@ -390,6 +398,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
   walk.tb = s_tb; walk.ro = s_ro; walk.nseg = p.nseg;
   for (int sg = 0; sg < 2; ++sg) {
     walk.nt[sg] = p.seg[sg].nt;
+    walk.mo[sg] = p.seg[sg].m_outer;
     walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
   }
   walk.seg = 0; walk.g = 0; walk.seg_first = 0;
@@ -559,7 +568,7 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // run fastest.  CTA `rank` of the pair owns m-tile 2*pair + rank of the group.
 struct PairWalker {
   const int32_t *tb, *ro, *pb;   // [2][kMaxExperts + 2] each: m-tile prefix, row offsets, pair prefix
-  int nt[2], G[2], nseg;
+  int nt[2], G[2], mo[2], nseg;
   int seg, g, seg_first;
   __device__ int seg_tiles(int s) const { return pb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
   __device__ int total() const {
@@ -582,8 +591,14 @@ struct PairWalker {
     const int local = local_seg - q[g] * n_t;
     t.seg = seg;
     t.g = g;
-    t.n_idx = local / np;
-    t.m_idx = 2 * (local - t.n_idx * np) + rank;
+    if (mo[seg]) {
+      const int pr = local / n_t;
+      t.n_idx = local - pr * n_t;
+      t.m_idx = 2 * pr + rank;
+    } else {
+      t.n_idx = local / np;
+      t.m_idx = 2 * (local - t.n_idx * np) + rank;
+    }
     t.prow0 = (b[g] + t.m_idx) * kTileM;
     t.urow0 = r[g] + t.m_idx * kTileM;
     t.valid = t.m_idx < b[g + 1] - b[g] ? min(kTileM, r[g + 1] - t.urow0) : 0;
@@ -667,6 +682,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   walk.tb = s_tb; walk.ro = s_ro; walk.pb = s_pb; walk.nseg = p.nseg;
   for (int sg = 0; sg < 2; ++sg) {
     walk.nt[sg] = p.seg[sg].nt;
+    walk.mo[sg] = p.seg[sg].m_outer;
     walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
   }
   walk.seg = 0; walk.g = 0; walk.seg_first = 0;
@@ -817,6 +833,13 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(uint4 *dst, const uint
   }
 }
 
+// Tile order of a single large group (the shared expert): when its rows [rows, k] are more than its weights
+// [w_rows, k] and too many to stay in L2 across a sweep over them, the n-tiles of one m-tile run fastest, so the
+// rows are read from DRAM once and the weights stay cached; otherwise the usual order.
+inline int rows_outweigh(int64_t rows, int64_t w_rows, int64_t k) {
+  return rows > w_rows && rows * k * 2 > ((int64_t)48 << 20);
+}
+
 constexpr size_t kSmemDyn = (size_t)STAGES * STAGE_BYTES + 1024;
 static_assert((size_t)STAGES2 * STAGE2_BYTES + 1024 == kSmemDyn, "both kernels use the same ring size");
 
@@ -852,6 +875,7 @@ pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const 
   p.plan = reinterpret_cast<DevPlan *>(reinterpret_cast<char *>(plan) + offsetof(DevPlan, status_router));
   Seg &S = p.seg[0];
   S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
+  S.m_outer = rows_outweigh(T, 2 * Fsh, H);
   p.nseg = 1;
   PCOMOE_CUDA_TRY(launch_pdl(kern, dim3(L->sm_count & ~1), dim3(kThreads), kSmemSide, st, mA, mB, mC, mA, mB, mC, p));
   count_launch();
@@ -917,6 +941,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
            make_map(&mC[ns], su, Fsh, H, 128);
       Seg &S = p.seg[ns++];
       S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
+      S.m_outer = rows_outweigh(T, 2 * Fsh, H);
     }
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; mC[1] = mC[0]; }
@@ -953,6 +978,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
       ok = ok && make_map(&mA[ns], Ush, (uint64_t)lay.t_pad, Fsh, kTileM) && make_map(&mB[ns], sd, H, Fsh, down_box);
       Seg &S = p.seg[ns++];
       S.G = 1; S.single_rows = T; S.nt = H / 256; S.kb = Fsh / BK; S.b_group_rows = 0;
+      S.m_outer = rows_outweigh(T, H, Fsh);
     }
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; }
