@@ -470,22 +470,26 @@ def main():
     R1 = int(stats[0])
     n_src = cfg.n - int(stats[4]); n_tgt = cfg.n - int(stats[5])
     work = algorithmic_work(cfg, R1, n_src, n_tgt)
-    stage_ms = {}
-    for name, fn in (("router", lambda: layer.router_logits(d_h)), ("route", lambda: layer.route(d_logits)), ("groups", lambda: layer.build_groups(cfg.T)),
-                     ("stage1_routed", lambda: layer.ffn_stages(d_h, 1)), ("stage1_shared", lambda: layer.ffn_stages(d_h, 2)),
-                     ("stage2_routed", lambda: layer.ffn_stages(d_h, 4)), ("stage2_shared", lambda: layer.ffn_stages(d_h, 8))):
-        if "shared" in name and not cfg.F_sh:
-            continue
-        if name == "router" and args.router < 0:
-            continue
-        ts = []
-        for i in range(3 + args.steps):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); fn(); b.record(stream)
-            torch.cuda.synchronize()
-            if i >= 3:
-                ts.append(a.elapsed_time(b))
-        stage_ms[name] = statistics.mean(ts)
+    # Stage times are taken inside a continuous run of steps (no idle gaps between the stages: the clocks and the
+    # cache state are those of the timed loop); every step goes stage by stage through the separate entry points
+    # with an event at each boundary.
+    stage_list = [("router", lambda: layer.router_logits(d_h)), ("route", lambda: layer.route(d_logits)),
+                  ("groups", lambda: layer.build_groups(cfg.T)),
+                  ("stage1_routed", lambda: layer.ffn_stages(d_h, 1)), ("stage1_shared", lambda: layer.ffn_stages(d_h, 2)),
+                  ("stage2_routed", lambda: layer.ffn_stages(d_h, 4)), ("stage2_shared", lambda: layer.ffn_stages(d_h, 8))]
+    stage_list = [(nm, fn) for nm, fn in stage_list
+                  if not ("shared" in nm and not cfg.F_sh) and not (nm == "router" and args.router < 0)]
+    n_rep = 3 + args.steps
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stage_list) + 1)] for _ in range(n_rep)]
+    torch.cuda.synchronize()
+    for i in range(n_rep):
+        marks[i][0].record(stream)
+        for j, (_, fn) in enumerate(stage_list):
+            fn()
+            marks[i][j + 1].record(stream)
+    torch.cuda.synchronize()
+    stage_ms = {nm: statistics.mean(marks[i][j].elapsed_time(marks[i][j + 1]) for i in range(3, n_rep))
+                for j, (nm, _) in enumerate(stage_list)}
     pk = peaks()
     tc_path = cfg.dtype == "bf16"
     if tc_path and cfg.T >= 1024:
