@@ -248,7 +248,8 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, co
 
 /* The whole hot path in one call: pcomoe_route_paths, pcomoe_build_path_groups and pcomoe_ffn_forward with the
  * same arguments and the same results.  What the single call adds: on prefill-sized batches of a tensor-core
- * layer with a shared expert, the shared expert's stage 1 (which depends on none of the routing) runs on a second
+ * layer with a shared expert, the shared expert's stage 1 (which depends on none of the routing; all of it, or the
+ * share of the tokens that fits the time) runs on a second
  * stream that the layer owns, beside the routing, grouping and row-gather kernels, and is joined before stage 2.
  * The second stream is ordered against `stream` with events on both sides, so the call behaves like work on
  * `stream` alone and can be recorded into a CUDA graph.  One call per layer at a time.  A wait that ran out in the

@@ -142,12 +142,12 @@ pcomoe_status launch_ffn_simt(const pcomoe_layer *L, int32_t T, const void *h, c
                               const void *sd, const pcomoe_groups *g, float *y, char *ws,
                               const WsLayout &lay, cudaStream_t st, int stages);
 pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const void *h, const void *sg,
-                                        const void *su, char *ws, const WsLayout &lay, cudaStream_t st);
+                                        const void *su, char *ws, const WsLayout &lay, cudaStream_t st, int32_t rows);
 pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                             const void *wu, const void *wd, const void *sg, const void *su,
                             const void *sd, const pcomoe_groups *g, float *y, char *ws,
                             const WsLayout &lay, cudaStream_t st, int stages,
-                            cudaEvent_t wait_before_stage2 = nullptr);
+                            cudaEvent_t wait_before_stage2 = nullptr, int32_t shared_row0 = 0);
 
 // bits of `stages`
 constexpr int kStage1Routed = 1, kStage1Shared = 2, kStage2Routed = 4, kStage2Shared = 8;

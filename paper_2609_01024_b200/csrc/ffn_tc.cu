@@ -853,7 +853,7 @@ constexpr int kSideStages = 4;
 constexpr size_t kSmemSide = (size_t)kSideStages * STAGE2_BYTES + 1024;
 
 pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const void *h, const void *sg,
-                                        const void *su, char *ws, const WsLayout &lay, cudaStream_t st) {
+                                        const void *su, char *ws, const WsLayout &lay, cudaStream_t st, int32_t rows) {
   const pcomoe_config &c = L->cfg;
   const int H = c.hidden, Fsh = c.shared_ffn;
   if (!L->tc_ok || Fsh <= 0) return PCOMOE_ERR_UNSUPPORTED;
@@ -867,15 +867,16 @@ pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const 
     attr_done = true;
   }
   CUtensorMap mA, mB, mC;
-  if (!(make_map(&mA, h, (uint64_t)T, H, kTileM) && make_map(&mB, sg, Fsh, H, 128) && make_map(&mC, su, Fsh, H, 128)))
+  // tokens [0, rows) only: the rest of the shared expert's stage 1 rides in the main stage-1 launch
+  if (!(make_map(&mA, h, (uint64_t)rows, H, kTileM) && make_map(&mB, sg, Fsh, H, 128) && make_map(&mC, su, Fsh, H, 128)))
     return PCOMOE_ERR_CUDA;
   TcParams p{};
   p.K = c.top_k; p.T = T; p.y = nullptr; p.ldy = H;
   // only the status word of the plan is touched by the kernel: point it at the router's word
   p.plan = reinterpret_cast<DevPlan *>(reinterpret_cast<char *>(plan) + offsetof(DevPlan, status_router));
   Seg &S = p.seg[0];
-  S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
-  S.m_outer = rows_outweigh(T, 2 * Fsh, H);
+  S.G = 1; S.single_rows = rows; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
+  S.m_outer = rows_outweigh(rows, 2 * Fsh, H);
   p.nseg = 1;
   PCOMOE_CUDA_TRY(launch_pdl(kern, dim3(L->sm_count & ~1), dim3(kThreads), kSmemSide, st, mA, mB, mC, mA, mB, mC, p));
   count_launch();
@@ -885,7 +886,8 @@ pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const 
 pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, const void *wg,
                             const void *wu, const void *wd, const void *sg, const void *su,
                             const void *sd, const pcomoe_groups *g, float *y, char *ws,
-                            const WsLayout &lay, cudaStream_t st, int stages, cudaEvent_t wait_before_stage2) {
+                            const WsLayout &lay, cudaStream_t st, int stages, cudaEvent_t wait_before_stage2,
+                            int32_t shared_row0) {
   const pcomoe_config &c = L->cfg;
   if (!L->tc_ok) return PCOMOE_ERR_UNSUPPORTED;
   const int n = c.n_experts, H = c.hidden, F = c.ffn, Fsh = c.shared_ffn;
@@ -937,11 +939,14 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
       S.path_w = merge ? reinterpret_cast<const float *>(ws + lay.path_wgt) : nullptr;
     }
     if (stages & kStage1Shared) {
-      ok = ok && make_map(&mA[ns], h, (uint64_t)T, H, kTileM) && make_map(&mB[ns], sg, Fsh, H, 128) &&
-           make_map(&mC[ns], su, Fsh, H, 128);
+      // tokens [shared_row0, T): the single-call forward runs the first tokens on its second stream
+      const int32_t rows = T - shared_row0;
+      ok = ok && make_map(&mA[ns], reinterpret_cast<const __nv_bfloat16 *>(h) + (size_t)shared_row0 * H, (uint64_t)rows, H, kTileM) &&
+           make_map(&mB[ns], sg, Fsh, H, 128) && make_map(&mC[ns], su, Fsh, H, 128);
       Seg &S = p.seg[ns++];
-      S.G = 1; S.single_rows = T; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0; S.u_out = Ush; S.ldu = Fsh;
-      S.m_outer = rows_outweigh(T, 2 * Fsh, H);
+      S.G = 1; S.single_rows = rows; S.nt = Fsh / 128; S.kb = H / BK; S.b_group_rows = 0;
+      S.u_out = Ush + (size_t)shared_row0 * Fsh; S.ldu = Fsh;
+      S.m_outer = rows_outweigh(rows, 2 * Fsh, H);
     }
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; mC[1] = mC[0]; }

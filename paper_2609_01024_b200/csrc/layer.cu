@@ -299,10 +299,23 @@ pcomoe_status pcomoe_layer_forward(const pcomoe_layer *L, int32_t T, const float
   // The shared expert's stage 1 needs nothing from routing, grouping and the row gather: on prefill-sized
   // batches it runs on the layer's second stream beside them and joins before stage 2.
   const bool overlap = tc && L->cfg.shared_ffn > 0 && use_cta_pairs(L, T);
+  int32_t side_rows = 0;
   if (overlap) {
+    // How many tokens of the shared expert the second stream takes: about as many as it can finish while the
+    // routing chain runs beside it (the chain runs at roughly half speed then); the rest joins the main stage-1
+    // launch, which has the deeper ring and one common tail.  Rough cost model in microseconds.
+    const pcomoe_config &c = L->cfg;
+    const double route_us = (double)T * L->n_active / 4.5e5;
+    const double gather_us = (double)T * c.top_k * 0.7 * c.hidden * 4.0 / 5.5e6;
+    const double chain_us = 2.0 * (route_us + 30.0 + gather_us);
+    const double side_us_per_token = 4.0 * c.hidden * c.shared_ffn / 1.35e9;
+    int64_t rows = (int64_t)(chain_us / side_us_per_token) / 256 * 256;
+    if (rows < 256) rows = 256;
+    if (rows > T || T - rows < 512) rows = T;
+    side_rows = (int32_t)rows;
     PCOMOE_CUDA_TRY(cudaEventRecord(L->ev_fork, st));
     PCOMOE_CUDA_TRY(cudaStreamWaitEvent(L->side_stream, L->ev_fork, 0));
-    s = launch_shared_stage1_side(L, T, d_h, d_wsh_gate, d_wsh_up, (char *)d_workspace, lay, L->side_stream);
+    s = launch_shared_stage1_side(L, T, d_h, d_wsh_gate, d_wsh_up, (char *)d_workspace, lay, L->side_stream, side_rows);
     // the join is recorded whatever happened, so that a stream capture always closes
     PCOMOE_CUDA_TRY(cudaEventRecord(L->ev_join, L->side_stream));
     if (s != PCOMOE_OK) {
@@ -317,7 +330,8 @@ pcomoe_status pcomoe_layer_forward(const pcomoe_layer *L, int32_t T, const float
     if (tc)
       s = launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down, groups,
                         (float *)d_y, (char *)d_workspace, lay, st,
-                        overlap ? (kStage1Routed | kStage2Routed | kStage2Shared) : 15, overlap ? L->ev_join : nullptr);
+                        !overlap ? 15 : side_rows < T ? 15 : (kStage1Routed | kStage2Routed | kStage2Shared),
+                        overlap ? L->ev_join : nullptr, side_rows);
     else
       s = launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down, groups,
                           (float *)d_y, (char *)d_workspace, lay, st, 15);
