@@ -41,6 +41,7 @@ SHAPES = [  # T, H, n, K, r, dtype, ffn_impl
     (33, 320, 10, 2, 0, "bf16", 0),       # H not a multiple of the 64-wide k-block: zero-filled tail
     (257, 256, 250, 2, 0, "bf16", 0),     # stacked tile at its 256-row limit
     (40, 128, 12, 3, 64, "bf16", 0),      # largest rank the tensor-core kernel takes
+    (50, 128, 128, 2, 64, "bf16", 0),     # n*r beyond the shared-memory copy of B_l: read from global memory
     (70, 256, 8, 2, 16, "bf16", 1),       # plain kernel, bf16
     (64, 256, 8, 2, 4, "f32", 0),         # fp32 layer: plain kernel
     (19, 200, 7, 2, 0, "f32", 0),
