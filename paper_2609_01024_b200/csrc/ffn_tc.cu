@@ -254,15 +254,43 @@ __device__ __forceinline__ void scatter_add_32x32(const TcParams &p, float *stag
 // Drains one accumulator (this thread's TMEM lane) and applies the stage's epilogue.  TMEM loads are issued
 // one step ahead of the arithmetic: a tcgen05.ld queues behind the MMAs already issued, so its latency is
 // long while the next tile is being computed, and must overlap the math and the stores of the previous step.
+// The stage-1 epilogue first lists the warp's (row, destination) pairs compactly in shared memory, so that the
+// write-out below runs over the destinations that exist (about 1.1-1.3 per row) instead of over the warp's maximum.
+constexpr int kDstList = 32 * kDstRegs;
+struct DstList {
+  int32_t *dst;      // [kDstList]
+  uint8_t *row;      // [kDstList]
+  float *w;          // [kDstList] (projection-side reuse only)
+};
+
 template <int STAGE, bool MERGE>
 __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, const TileInfo &t, const RowCtx &c,
-                                              uint32_t taddr, float *stage) {
+                                              uint32_t taddr, float *stage, const DstList dl) {
   if (STAGE == 1) {
     // 32 rows x 64 bf16 columns are collected in shared memory, then every destination row receives its
     // 128 contiguous bytes from eight lanes (whole lines), four rows per instruction.
     const int lane = threadIdx.x & 31;
     const size_t col0 = (size_t)t.n_idx * 128;
-    const int max_nd = c.dst_in_regs ? __reduce_max_sync(0xffffffffu, c.nd) : 0;
+    int n_dst = 0;
+    {
+      const int nd = c.dst_in_regs ? c.nd : 0;
+      int incl = nd;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      n_dst = __shfl_sync(0xffffffffu, incl, 31);
+      const int base = incl - nd;
+#pragma unroll
+      for (int j = 0; j < kDstRegs; ++j)
+        if (j < nd) {
+          dl.dst[base + j] = c.dst[j];
+          dl.row[base + j] = (uint8_t)lane;
+          if (MERGE) dl.w[base + j] = c.wsc[j];
+        }
+      __syncwarp();
+    }
     unsigned char *srow = reinterpret_cast<unsigned char *>(stage) + lane * (kEpiStride * 4);
     uint32_t g0[32], u0[32], g1[32], u1[32];
     tmem_ld32_issue(taddr, g0);
@@ -289,25 +317,15 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
 #pragma unroll
       for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow + 64)[q] = out[q];
       __syncwarp();
-      for (int k = 0; k < max_nd; ++k) {
-        int dk = -1;
-        float wk = 0.0f;
-#pragma unroll
-        for (int j = 0; j < kDstRegs; ++j)
-          if (j == k && k < c.nd) {
-            dk = c.dst[j];
-            if (MERGE) wk = c.wsc[j];
-          }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int row = i * 4 + (lane >> 3);
-          const int d = __shfl_sync(0xffffffffu, dk, row);
-          const float sc = MERGE ? __shfl_sync(0xffffffffu, wk, row) : 0.0f;
+      for (int e0 = 0; e0 < n_dst; e0 += 4) {
+        const int e = e0 + (lane >> 3);
+        if (e < n_dst) {
+          const int row = dl.row[e], d = dl.dst[e];
           const uint4 x = *reinterpret_cast<const uint4 *>(reinterpret_cast<unsigned char *>(stage) +
                                                            row * (kEpiStride * 4) + (lane & 7) * 16);
           if (d >= 0) *reinterpret_cast<uint4 *>(S.u_out + (size_t)d * S.ldu + col0 + c0 + (lane & 7) * 8) = x;
           else if (MERGE && d <= -2)
-            red_add_scaled_bf16x8(S.u_out + (size_t)(-d - 2) * S.ldu + col0 + c0 + (lane & 7) * 8, x, sc);
+            red_add_scaled_bf16x8(S.u_out + (size_t)(-d - 2) * S.ldu + col0 + c0 + (lane & 7) * 8, x, dl.w[e]);
         }
       }
       __syncwarp();
@@ -349,6 +367,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ __align__(16) float s_epi[4 * 32 * kEpiStride];   // per epilogue warp: 32 rows being turned around
+  __shared__ int32_t s_dl_dst[STAGE == 1 ? 4 * kDstList : 1];
+  __shared__ uint8_t s_dl_row[STAGE == 1 ? 4 * kDstList : 1];
+  __shared__ float s_dl_w[(STAGE == 1 && MERGE) ? 4 * kDstList : 1];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;   // 1024-byte aligned for the swizzle
@@ -483,7 +504,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
       epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
-                           s_epi + (warp - 2) * 32 * kEpiStride);
+                           s_epi + (warp - 2) * 32 * kEpiStride,
+                           DstList{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0),
+                                   s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
+                                   s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)});
       tc_fence_before();
       mbar_arrive(acce_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -619,6 +643,9 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ __align__(16) float s_epi[4 * 32 * kEpiStride];   // per epilogue warp: 32 rows being turned around
+  __shared__ int32_t s_dl_dst[STAGE == 1 ? 4 * kDstList : 1];
+  __shared__ uint8_t s_dl_row[STAGE == 1 ? 4 * kDstList : 1];
+  __shared__ float s_dl_w[(STAGE == 1 && MERGE) ? 4 * kDstList : 1];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
@@ -770,7 +797,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
       epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
-                           s_epi + (warp - 2) * 32 * kEpiStride);
+                           s_epi + (warp - 2) * 32 * kEpiStride,
+                           DstList{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0),
+                                   s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
+                                   s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)});
       tc_fence_before();
       mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));   // the leader's MMA waits for both halves
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
