@@ -30,7 +30,6 @@ constexpr uint32_t ACC_COLS = 256;                  // fp32 accumulator columns 
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int kThreads = 192;
 constexpr int kEpiStride = 36;               // words per row staged by the epilogue: 16-byte aligned, conflict-free
-constexpr int kDstRegs = 8;                 // stage-1 epilogue keeps up to this many destinations in registers
 
 // One run of tiles that share tensor maps, k-loop length and epilogue parameters: the routed groups, or
 // the shared expert (a single group whose rows are the tokens themselves).
@@ -128,6 +127,15 @@ struct TileWalker {
   }
 };
 
+// The stage-1 epilogue first lists the warp's (row, destination) pairs compactly in shared memory, so that the
+// write-out below runs over the destinations that exist (about 1.1-1.3 per row) instead of over the warp's maximum.
+constexpr int kDstList = 256;                // entries per epilogue warp (32 rows x up to 8 destinations)
+struct DstList {
+  int32_t *dst;      // [kDstList]
+  uint8_t *row;      // [kDstList]
+  float *w;          // [kDstList] (projection-side reuse only)
+};
+
 // What an epilogue thread needs to know about its row, looked up before the accumulator is ready so that
 // the loads overlap the MMAs.
 struct RowCtx {
@@ -135,21 +143,18 @@ struct RowCtx {
   int token;
   float wgt;          // stage 2: path weight
   int my_prow;        // padded row of this thread
-  int nd;             // stage 1, routed: number of stage-2 rows fed by this (token, source) slot
-  int dst[kDstRegs];  //                  and those rows (when K <= kDstRegs)
-  float wsc[kDstRegs];//                  weight of the path behind each destination (projection-side reuse only)
-  bool dst_in_regs;
+  int n_dst;          // stage 1: entries of the warp's destination list; -1: too many for the list, look up on the spot
 };
 
 template <int STAGE, bool MERGE>
-__device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, const TileInfo &t, int r) {
+__device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, const TileInfo &t, int r, const DstList dl) {
   RowCtx c;
+  const int lane = threadIdx.x & 31;
   const bool valid = r < t.valid;
   c.token = 0;
   c.wgt = 0.0f;
   c.my_prow = t.prow0 + r;
-  c.nd = 0;
-  c.dst_in_regs = p.K <= kDstRegs || !S.row_token;   // the same for every lane of the warp
+  c.n_dst = 0;
   if (STAGE == 1) {
     if (valid && S.row_token) c.token = S.row_token[c.my_prow];
   } else if (valid) {
@@ -159,25 +164,40 @@ __device__ __forceinline__ RowCtx prepare_row(const TcParams &p, const Seg &S, c
   }
   c.ok = valid && (unsigned)c.token < (unsigned)p.T;
   if (valid && !c.ok) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_INDEX);
-  if (STAGE == 1 && c.ok && !S.row_token) {   // shared expert: the row is its own destination
-    c.dst[0] = c.my_prow;
-    c.nd = 1;
-  }
-  if (STAGE == 1 && c.ok && S.row_token && c.dst_in_regs) {
-#pragma unroll
-    for (int k = 0; k < kDstRegs; ++k) {
-      if (k < p.K && S.path_prow1[(size_t)c.token * p.K + k] == c.my_prow) {
-        const int d = S.path_pos2[(size_t)c.token * p.K + k];
-        const float wk = MERGE ? S.path_w[(size_t)c.token * p.K + k] : 0.0f;
-#pragma unroll
-        for (int j = 0; j < kDstRegs; ++j)
-          if (j == c.nd) {
-            c.dst[j] = d;
-            if (MERGE) c.wsc[j] = wk;
-          }
-        ++c.nd;
+  if (STAGE == 1) {
+    // the warp's (row, destination) pairs, compacted with ballots: a (token, source) slot feeds every path of the
+    // token that has this source (Sec. 4.3 reuse); a row of the shared expert feeds itself
+    const unsigned below = (1u << lane) - 1u;
+    if (!S.row_token) {
+      const unsigned m = __ballot_sync(0xffffffffu, c.ok);
+      if (c.ok) {
+        const int pos = __popc(m & below);
+        dl.dst[pos] = c.my_prow;
+        dl.row[pos] = (uint8_t)lane;
       }
+      c.n_dst = __popc(m);
+    } else {
+      int base = 0;
+      const size_t q0 = (size_t)c.token * p.K;
+      for (int k = 0; k < p.K; ++k) {
+        const bool hit = c.ok && S.path_prow1[q0 + k] == c.my_prow;
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        const int n_hit = __popc(m);
+        if (base + n_hit > kDstList) {   // the same decision in every lane
+          base = -1;
+          break;
+        }
+        if (hit) {
+          const int pos = base + __popc(m & below);
+          dl.dst[pos] = S.path_pos2[q0 + k];
+          dl.row[pos] = (uint8_t)lane;
+          if (MERGE) dl.w[pos] = S.path_w[q0 + k];
+        }
+        base += n_hit;
+      }
+      c.n_dst = base;
     }
+    __syncwarp();
   }
   return c;
 }
@@ -254,15 +274,6 @@ __device__ __forceinline__ void scatter_add_32x32(const TcParams &p, float *stag
 // Drains one accumulator (this thread's TMEM lane) and applies the stage's epilogue.  TMEM loads are issued
 // one step ahead of the arithmetic: a tcgen05.ld queues behind the MMAs already issued, so its latency is
 // long while the next tile is being computed, and must overlap the math and the stores of the previous step.
-// The stage-1 epilogue first lists the warp's (row, destination) pairs compactly in shared memory, so that the
-// write-out below runs over the destinations that exist (about 1.1-1.3 per row) instead of over the warp's maximum.
-constexpr int kDstList = 32 * kDstRegs;
-struct DstList {
-  int32_t *dst;      // [kDstList]
-  uint8_t *row;      // [kDstList]
-  float *w;          // [kDstList] (projection-side reuse only)
-};
-
 template <int STAGE, bool MERGE>
 __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, const TileInfo &t, const RowCtx &c,
                                               uint32_t taddr, float *stage, const DstList dl) {
@@ -271,26 +282,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
     // 128 contiguous bytes from eight lanes (whole lines), four rows per instruction.
     const int lane = threadIdx.x & 31;
     const size_t col0 = (size_t)t.n_idx * 128;
-    int n_dst = 0;
-    {
-      const int nd = c.dst_in_regs ? c.nd : 0;
-      int incl = nd;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const int o = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += o;
-      }
-      n_dst = __shfl_sync(0xffffffffu, incl, 31);
-      const int base = incl - nd;
-#pragma unroll
-      for (int j = 0; j < kDstRegs; ++j)
-        if (j < nd) {
-          dl.dst[base + j] = c.dst[j];
-          dl.row[base + j] = (uint8_t)lane;
-          if (MERGE) dl.w[base + j] = c.wsc[j];
-        }
-      __syncwarp();
-    }
+    const int n_dst = c.n_dst;
     unsigned char *srow = reinterpret_cast<unsigned char *>(stage) + lane * (kEpiStride * 4);
     uint32_t g0[32], u0[32], g1[32], u1[32];
     tmem_ld32_issue(taddr, g0);
@@ -303,7 +295,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
       tmem_ld32_issue(taddr + c0 + 32, g1);
       tmem_ld32_issue(taddr + 128 + c0 + 32, u1);
       swiglu_pack32(g0, u0, out);
-      if (c.ok && !c.dst_in_regs) store_row_lookup<MERGE>(p, S, c, col0 + c0, out);
+      if (c.ok && n_dst < 0) store_row_lookup<MERGE>(p, S, c, col0 + c0, out);
 #pragma unroll
       for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow)[q] = out[q];
       tmem_wait_ld();
@@ -313,7 +305,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams &p, const Seg &S, c
         tmem_ld32_issue(taddr + 128 + c0 + 64, u0);
       }
       swiglu_pack32(g1, u1, out);
-      if (c.ok && !c.dst_in_regs) store_row_lookup<MERGE>(p, S, c, col0 + c0 + 32, out);
+      if (c.ok && n_dst < 0) store_row_lookup<MERGE>(p, S, c, col0 + c0 + 32, out);
 #pragma unroll
       for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(srow + 64)[q] = out[q];
       __syncwarp();
@@ -500,14 +492,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
       const TileInfo t = walk.at(tile);
       const Seg &S = p.seg[t.seg];
-      const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r);
+      const DstList dl{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0), s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
+                       s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)};
+      const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r, dl);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
       epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
-                           s_epi + (warp - 2) * 32 * kEpiStride,
-                           DstList{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0),
-                                   s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
-                                   s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)});
+                           s_epi + (warp - 2) * 32 * kEpiStride, dl);
       tc_fence_before();
       mbar_arrive(acce_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -793,14 +784,13 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
     for (int tile = pair_id; tile < total; tile += n_pairs) {
       const TileInfo t = walk.at(tile, rank);
       const Seg &S = p.seg[t.seg];
-      const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r);
+      const DstList dl{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0), s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
+                       s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)};
+      const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r, dl);
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
       tc_fence_after();
       epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
-                           s_epi + (warp - 2) * 32 * kEpiStride,
-                           DstList{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0),
-                                   s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
-                                   s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)});
+                           s_epi + (warp - 2) * 32 * kEpiStride, dl);
       tc_fence_before();
       mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));   // the leader's MMA waits for both halves
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }

@@ -163,6 +163,25 @@ def test_cuda_graph_replay_matches_eager(G, oracle):
 
 
 @pytest.mark.parametrize("impl", [2, 3])
+def test_one_source_feeding_many_paths_per_token(G, oracle, impl):
+    """K = 12 paths per token, all with the same source: every stage-1 row feeds 12 stage-2 rows, more per warp than
+    the epilogue's destination list holds, so the rows are stored by looking their destinations up on the spot."""
+    import torch
+    cfg = wl.small_case(92, T=300, H=256, F=128, n=16, K=12, mask_p=1.0)
+    L = wl.make_layer(cfg)
+    z = L.logits.copy()
+    z[:, 5] += 100.0
+    layer = G.make_gpu_layer(cfg, L, ffn_impl=impl)
+    y = layer.forward(torch.from_numpy(z).to(layer.device), G.B.to_device(L.h)).cpu().numpy()
+    assert layer.device_status() == 0
+    rs, rt, rw = oracle.route(z, L.mask, L.bias, cfg.lam, cfg.K)
+    assert np.all(rs == 5)
+    assert np.array_equal(layer.path_tgt[:cfg.T].cpu().numpy(), rt)
+    assert layer.groups.to_host()["R1"] == cfg.T
+    G.check_output(y, oracle.ffn(wl.hidden_as_f32(cfg, L.h), L.w_gate, L.w_up, L.w_down, rs, rt, rw))
+
+
+@pytest.mark.parametrize("impl", [2, 3])
 def test_every_token_on_one_source(G, oracle, impl):
     """Degenerate load: one expert's logit dominates, so every path of every token has the same source - a single
     stage-1 group of T rows (several tiles and a ragged tail), all other source groups empty."""
