@@ -482,6 +482,7 @@ def main():
     n_rep = 3 + args.steps
     marks = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stage_list) + 1)] for _ in range(n_rep)]
     torch.cuda.synchronize()
+    time.sleep(1.0)        # start from the idle power state the headline loop started from
     for i in range(n_rep):
         marks[i][0].record(stream)
         for j, (_, fn) in enumerate(stage_list):
