@@ -935,6 +935,19 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   }
   const bool pair = use_cta_pairs(L, T);
   const int grid = pair ? (L->sm_count & ~1) : L->sm_count;
+  // Decode-sized batches (every group at most one 128-row tile): the tile count is known up front, and a grid that
+  // divides it evenly avoids a last wave in which a handful of CTAs stream their weights alone at a fraction of the
+  // HBM rate (Mixtral shape: 896 stage-1 tiles run as 7 waves of 128 CTAs instead of 6 waves of 148 plus 8 tiles).
+  auto even_grid = [&](int64_t tiles) {
+    if (pair || (int64_t)T * c.top_k > kTileM || tiles <= 0) return grid;
+    const int64_t waves = (tiles + grid - 1) / grid;
+    return (int)((tiles + waves - 1) / waves);
+  };
+  const int mt_sh = (T + kTileM - 1) / kTileM;
+  const int grid1 = even_grid(((stages & kStage1Routed) ? (int64_t)n * (F / 128) : 0) +
+                              ((stages & kStage1Shared) ? (int64_t)mt_sh * (Fsh / 128) : 0));
+  const int grid2 = even_grid(((stages & kStage2Routed) ? (int64_t)n * (H / 256) : 0) +
+                              ((stages & kStage2Shared) ? (int64_t)mt_sh * (H / 256) : 0));
   const bool merge = c.target_reuse != 0;
   const uint32_t down_box = pair ? 128 : 256;   // a CTA of a pair loads half of the 256-row slice of W_down
 
@@ -977,7 +990,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     }
     auto k3 = merge ? (pair ? grouped_gemm_pair_kernel<1, true> : grouped_gemm_kernel<1, true>)
                     : (pair ? grouped_gemm_pair_kernel<1, false> : grouped_gemm_kernel<1, false>);
-    PCOMOE_CUDA_TRY(launch_pdl(k3, dim3(grid), dim3(kThreads), kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
+    PCOMOE_CUDA_TRY(launch_pdl(k3, dim3(grid1), dim3(kThreads), kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
     count_launch();
   }
 
@@ -1008,7 +1021,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
     if (!ok) return PCOMOE_ERR_CUDA;
     if (ns == 1) { mA[1] = mA[0]; mB[1] = mB[0]; }
     p.nseg = ns;
-    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<2> : grouped_gemm_kernel<2>, dim3(grid), dim3(kThreads),
+    PCOMOE_CUDA_TRY(launch_pdl(pair ? grouped_gemm_pair_kernel<2> : grouped_gemm_kernel<2>, dim3(grid2), dim3(kThreads),
                                kSmemDyn, st, mA[0], mB[0], mB[0], mA[1], mB[1], mB[1], p));
     count_launch();
   }
