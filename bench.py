@@ -33,7 +33,7 @@ METRIC = "path_moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 # DRAM bytes (dram__bytes_read + dram__bytes_write) of ONE launch of the dominant kernel (stage-1 grouped GEMM) on
 # the benchmark layers, from the ncu capture summarised in profiles/kernels_per_config.md
-NCU_TRAFFIC_STAGE1 = {2: 2321.7e6, 3: 1119.4e6, 4: 1257.2e6, 5: 1891.6e6}   # routed groups only (the launch the stage-1 time is taken from)
+NCU_TRAFFIC_STAGE1 = {2: 2321.7e6, 3: 1119.4e6, 4: 1257.2e6, 5: 1890.9e6}   # routed groups only (the launch the stage-1 time is taken from)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
