@@ -64,7 +64,8 @@ typedef struct {
   int32_t ffn;          /* F, per-expert intermediate width                                   */
   int32_t shared_ffn;   /* F_sh, width of the always-on shared expert; 0 = none               */
   int32_t in_dtype;     /* pcomoe_dtype of h and of every weight                              */
-  int32_t out_dtype;    /* pcomoe_dtype of y; only PCOMOE_FP32 is implemented                 */
+  int32_t out_dtype;    /* pcomoe_dtype of y.  PCOMOE_BF16: y is accumulated in fp32 (in the
+                           workspace) and rounded to nearest-even once, after the last addition  */
   float lambda;         /* scale of the target-side prior in the path score (Sec. 4.2)        */
   int32_t norm_topk;    /* 1: beta = softmax over the K selected scores;
                            0: softmax over the whole active set, gathered at the K selected   */
@@ -199,10 +200,16 @@ pcomoe_status pcomoe_build_path_groups(const pcomoe_layer *layer, int32_t T,
  *
  * Limits and rules:
  *   - The layer must have been created on the current device (else INVALID_ARG).
- *   - The scratch need grows with T*K and n; T*K <= 65536 always fits (n <= 256).  A larger batch
- *     that does not fit is refused with PCOMOE_ERR_SHAPE and nothing is enqueued.
+ *   - The scratch need grows with T*K, n and the number of SMs: what must fit is everything the
+ *     grouping kernels keep in a workspace (per-block histograms 8*n*NB bytes with NB <= max(4*SMs,
+ *     T/32) blocks, the tile prefixes, and 12 bytes per path plus 4 bytes per padded stage-1 row).
+ *     On a GPU of up to 256 SMs every batch with T*K <= 65536 fits for every n <= 256 (the largest
+ *     need, n = 256, K = 1, 148 SMs, is 2 135 296 bytes).  A batch that does not fit is refused with
+ *     PCOMOE_ERR_SHAPE and nothing is enqueued.
  *   - The first call on a device looks up the array's device address (a one-time set-up for that
- *     device); make that first call before any stream capture begins.
+ *     device).  The array is part of the library's device image, and the driver may load that part of
+ *     the image - and so claim the array's memory - only at this first look-up: make the first call at
+ *     start-up, while device memory is still available, and before any stream capture begins.
  *   - Every call on a device uses the same array.  Each call zero-fills what must start from zero,
  *     so nothing is carried over from the previous call, but two calls that can run on the GPU at
  *     the same time (different streams) race: serialise them.
@@ -210,7 +217,7 @@ pcomoe_status pcomoe_build_path_groups(const pcomoe_layer *layer, int32_t T,
  * the internal status word only (not readable through pcomoe_device_status); rows of an
  * out-of-range expert id are skipped.
  */
-#define PCOMOE_STATIC_SCRATCH_BYTES (2u << 20)
+#define PCOMOE_STATIC_SCRATCH_BYTES (3u << 20)
 pcomoe_status pcomoe_build_path_groups_static(const pcomoe_layer *layer, int32_t T,
                                               const int32_t *d_path_src, const int32_t *d_path_tgt,
                                               const float *d_path_w, const pcomoe_groups *out,
@@ -224,8 +231,9 @@ pcomoe_status pcomoe_build_path_groups_static(const pcomoe_layer *layer, int32_t
  *            y[s2_token[q],:] += s2_w[q] * W_down^(j) U[s2_s1row[q],:]   (fp32 accumulate and add)
  *   shared   y[t,:] += Wsh_down (SiLU(Wsh_gate h_t) (.) (Wsh_up h_t))  when F_sh > 0 (weight 1).
  *   d_h [T,H]; d_w_gate, d_w_up [n,F,H]; d_w_down [n,H,F]; shared weights or NULL (all in in_dtype);
- *   d_y [T,H] fp32, fully overwritten (zero-filled first, then accumulated with atomic adds, so the
- *   order of the additions - and the last bits of y - can differ between calls).
+ *   d_y [T,H] in out_dtype, fully overwritten (the fp32 sum is zero-filled first, then accumulated with
+ *   atomic adds, so the order of the additions - and the last bits of y - can differ between calls; a
+ *   bf16 y is that fp32 sum, kept in the workspace, rounded once at the end).
  * `groups` and d_workspace must come from pcomoe_build_path_groups for the same T.
  * Errors: INVALID_ARG, SHAPE, WORKSPACE, UNSUPPORTED, CUDA.  Device: TIMEOUT, INDEX.
  */
@@ -262,6 +270,36 @@ pcomoe_status pcomoe_layer_forward(const pcomoe_layer *layer, int32_t T, const f
                                    int32_t *d_path_tgt, float *d_path_w, const pcomoe_groups *groups, void *d_y,
                                    void *d_workspace, size_t ws_bytes, void *stream);
 
+/* The single call from HOST buffers (Sec. 4.1 layer output, Sec. 4.3 execution; same results as
+ * pcomoe_layer_forward).  A pipe owns what a stream of batches living in host memory needs: device copies of
+ * the inputs and of y in `slots` slots, the path and group arrays, the workspace, a copy-in stream, a compute
+ * stream and a copy-out stream.  pcomoe_host_pipe_submit enqueues, for one batch, the host->device copies of
+ * logits and hidden states, the whole hot path, and the device->host copy of y, each on its own stream and
+ * ordered by events, so that with slots >= 2 the copies of neighbouring batches overlap the kernels.  It never
+ * blocks the host; the host buffers of a batch must stay valid, and h_y must not be read, until
+ * pcomoe_host_pipe_wait has returned.  Copies from or to pageable host memory work but are staged by the
+ * driver: pass page-locked (pinned) buffers for overlap.
+ *   create   allocates the device memory (the only call of the three that does), for batches of up to
+ *            max_tokens, 1 <= slots <= 4.  The device weight pointers (as in pcomoe_ffn_forward) are kept, not
+ *            copied, and must outlive the pipe.  Must be called with the layer's device current.
+ *   submit   h_logits [T,n] fp32, h_tgt_logits [T,n] fp32 or NULL, h_hidden [T,H] in_dtype, h_y [T,H] out_dtype
+ *            (host pointers).  T = 0 is a no-op.
+ *   wait     blocks until every submitted batch is complete and returns the first device-side error any of
+ *            them recorded (TIMEOUT, INDEX), else OK.
+ *   groups / paths  device arrays of the most recent batch (valid after wait), for inspection.
+ * Errors: INVALID_ARG, SHAPE (T < 0 or T > max_tokens, slots out of range), CUDA, and those of the hot calls. */
+typedef struct pcomoe_host_pipe pcomoe_host_pipe;
+pcomoe_status pcomoe_host_pipe_create(const pcomoe_layer *layer, int32_t max_tokens, int32_t slots,
+                                      const void *d_w_gate, const void *d_w_up, const void *d_w_down,
+                                      const void *d_wsh_gate, const void *d_wsh_up, const void *d_wsh_down,
+                                      pcomoe_host_pipe **out);
+pcomoe_status pcomoe_host_pipe_submit(pcomoe_host_pipe *pipe, int32_t T, const float *h_logits,
+                                      const float *h_tgt_logits, const void *h_hidden, void *h_y);
+pcomoe_status pcomoe_host_pipe_wait(pcomoe_host_pipe *pipe);
+pcomoe_status pcomoe_host_pipe_arrays(const pcomoe_host_pipe *pipe, pcomoe_groups *groups, int32_t **d_path_src,
+                                      int32_t **d_path_tgt, float **d_path_w);
+pcomoe_status pcomoe_host_pipe_destroy(pcomoe_host_pipe *pipe);
+
 /* Router in front of the path gate (Sec. 3.1: the router maps a token's hidden state to routing scores;
  * Sec. 4.2 uses them as the base routing signal g_base(h), and as g_tgt(h) unless a second head is given):
  *     d_logits[t,e] = sum_k d_h[t,k] * d_w_router[e,k]
@@ -296,6 +334,22 @@ pcomoe_status pcomoe_residual_cast(const pcomoe_layer *layer, int32_t T, const v
  * recorded (PCOMOE_OK if none): the layer's word is cleared by the next pcomoe_build_path_groups, the
  * router's by this call once it has been read. */
 pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream);
+
+/* Failure detection on the device.  Every wait of the tensor-core kernels (on an mbarrier that a TMA copy, an MMA
+ * or the partner CTA completes) is bounded: when the limit runs out the CTA records PCOMOE_ERR_TIMEOUT in the
+ * workspace's status word, lets its copies land, frees its tensor memory and returns, so the context stays usable
+ * and pcomoe_device_status reports the failure.  (The paper has no counterpart; its engine is not described at
+ * this level.)
+ *   pcomoe_set_wait_limit_us   sets the limit for kernels launched afterwards, process-wide; 0 restores the
+ *                              default of 2 s; more than 60 s is INVALID_ARG.
+ *   pcomoe_selftest_wait_timeout  enqueues a one-warp kernel that waits, with the same routine and limit, on a
+ *                              barrier nothing will complete (no copy or MMA is involved), and so ends through the
+ *                              give-up path: afterwards pcomoe_device_status(d_workspace) returns TIMEOUT, and the
+ *                              next pcomoe_build_path_groups on that workspace clears the word again.  d_workspace
+ *                              needs room for the status header only (256 bytes, 256-byte aligned).
+ * Errors: INVALID_ARG, WORKSPACE, CUDA. */
+pcomoe_status pcomoe_set_wait_limit_us(uint32_t limit_us);
+pcomoe_status pcomoe_selftest_wait_timeout(void *d_workspace, void *stream);
 
 /* Launch counters (kernels and memsets enqueued by this library since load, per process). */
 int64_t pcomoe_launch_count(void);

@@ -93,6 +93,10 @@ static int cand_cmp(const void *pa, const void *pb) {
  *            times routed_scale.
  * z = g_base [T,n], u = g_tgt [T,n] (pass z again when there is one router).
  * Outputs are rank ordered: src, tgt [T,K] int32; w [T,K] fp32; score [T,K] fp32 (optional).
+ * The paper assumes finite routing signals.  Reading for the rest: a path whose score is NaN or infinite
+ * (a router that masks an expert with a -inf logit, an overflow) is not eligible for that token - the same
+ * thing the mask does to a path, "prior to gating" (Sec. 4.2) - and a token left with fewer than K eligible
+ * paths gets src = tgt = -1 and weight 0 in the ranks it cannot fill.
  * ------------------------------------------------------------------------- */
 int pcomoe_oracle_route(int32_t T, int32_t n, int32_t K, const float *z, const float *u,
                         const uint8_t *M, const float *B, float lambda, int32_t norm_topk,
@@ -119,16 +123,25 @@ int pcomoe_oracle_route(int32_t T, int32_t n, int32_t K, const float *z, const f
           float b = lambda * u[(size_t)t * n + j];               /* rounded */
           float s = a + b;                                       /* rounded */
           s = s + 0.0f;                                          /* -0 -> +0 */
+          if (!isfinite(s)) continue; /* a NaN or infinite score takes the path out of this token's active set */
           c[cnt].s = s;
           c[cnt].flat = i * n + j;
           ++cnt;
         }
       qsort(c, (size_t)cnt, sizeof(cand_t), cand_cmp);
+      const int32_t live = cnt < K ? cnt : K; /* fewer than K finite scores: the remaining ranks stay empty */
+      for (int32_t k = live; k < K; ++k) {
+        src[(size_t)t * K + k] = -1;
+        tgt[(size_t)t * K + k] = -1;
+        w[(size_t)t * K + k] = 0.0f;
+        if (score) score[(size_t)t * K + k] = -INFINITY;
+      }
+      if (live == 0) continue;
       double s0 = (double)c[0].s;
       double den = 0.0;
-      int32_t lim = norm_topk ? K : cnt;
+      int32_t lim = norm_topk ? live : cnt;
       for (int32_t a = 0; a < lim; ++a) den += exp((double)c[a].s - s0);
-      for (int32_t k = 0; k < K; ++k) {
+      for (int32_t k = 0; k < live; ++k) {
         src[(size_t)t * K + k] = c[k].flat / n;
         tgt[(size_t)t * K + k] = c[k].flat % n;
         double beta = exp((double)c[k].s - s0) / den * (double)routed_scale;

@@ -23,7 +23,9 @@ PCOMOE_FFN_AUTO, PCOMOE_FFN_SIMT, PCOMOE_FFN_TCGEN05, PCOMOE_FFN_TCGEN05_PAIR = 
 EXPORTS = ["pcomoe_mask_from_bias", "pcomoe_mask_tighten", "pcomoe_layer_create", "pcomoe_layer_destroy", "pcomoe_layer_active_set", "pcomoe_workspace_bytes",
            "pcomoe_route_paths", "pcomoe_build_path_groups", "pcomoe_build_path_groups_static", "pcomoe_ffn_forward",
            "pcomoe_ffn_forward_stages", "pcomoe_layer_forward", "pcomoe_router_logits", "pcomoe_residual_cast",
-           "pcomoe_device_status",
+           "pcomoe_host_pipe_create", "pcomoe_host_pipe_submit", "pcomoe_host_pipe_wait", "pcomoe_host_pipe_arrays",
+           "pcomoe_host_pipe_destroy",
+           "pcomoe_device_status", "pcomoe_set_wait_limit_us", "pcomoe_selftest_wait_timeout",
            "pcomoe_launch_count", "pcomoe_status_string"]
 
 
@@ -74,6 +76,14 @@ def load_library(path: str | None = None):
     lib.pcomoe_router_logits.argtypes = [vp, i32, vp, vp, vp, vp, i32, ctypes.c_float, vp, vp, sz, vp]
     lib.pcomoe_residual_cast.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.pcomoe_device_status.argtypes = [vp, vp]
+    lib.pcomoe_host_pipe_create.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.POINTER(vp)]
+    lib.pcomoe_host_pipe_submit.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.pcomoe_host_pipe_wait.argtypes = [vp]
+    lib.pcomoe_host_pipe_arrays.argtypes = [vp, ctypes.POINTER(pcomoe_groups), ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                            ctypes.POINTER(vp)]
+    lib.pcomoe_host_pipe_destroy.argtypes = [vp]
+    lib.pcomoe_set_wait_limit_us.argtypes = [ctypes.c_uint32]
+    lib.pcomoe_selftest_wait_timeout.argtypes = [vp, vp]
     lib.pcomoe_launch_count.restype = ctypes.c_int64
     lib.pcomoe_status_string.restype = ctypes.c_char_p
     lib.pcomoe_status_string.argtypes = [i32]
@@ -249,18 +259,26 @@ def pcomoe_device_status(workspace) -> int:
     return int(load_library().pcomoe_device_status(_ptr(workspace), _stream()))
 
 
+def pcomoe_set_wait_limit_us(limit_us: int):
+    _check(load_library().pcomoe_set_wait_limit_us(int(limit_us)), "pcomoe_set_wait_limit_us")
+
+
+def pcomoe_selftest_wait_timeout(workspace):
+    _check(load_library().pcomoe_selftest_wait_timeout(_ptr(workspace), _stream()), "pcomoe_selftest_wait_timeout")
+
+
 class PathMoELayer:
     """Owns the device buffers of one layer and chains the three hot calls.  Marshalling only."""
 
     def __init__(self, *, n_experts, top_k, hidden, ffn, mask, bias, w_gate, w_up, w_down, shared=None,
-                 max_tokens, in_dtype=PCOMOE_BF16, lam=0.5, norm_topk=1, routed_scale=1.0, dedup=1,
-                 ffn_impl=PCOMOE_FFN_AUTO, target_reuse=0, device="cuda:0"):
+                 max_tokens, in_dtype=PCOMOE_BF16, out_dtype=PCOMOE_FP32, lam=0.5, norm_topk=1, routed_scale=1.0,
+                 dedup=1, ffn_impl=PCOMOE_FFN_AUTO, target_reuse=0, device="cuda:0"):
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self.n, self.K, self.H, self.F = n_experts, top_k, hidden, ffn
         self.F_sh = 0 if shared is None or shared[0] is None else int(shared[0].shape[0])
         self.layer = pcomoe_layer_create(n_experts=n_experts, top_k=top_k, hidden=hidden, ffn=ffn, mask=mask,
-                                         bias=bias, shared_ffn=self.F_sh, in_dtype=in_dtype, lam=lam,
+                                         bias=bias, shared_ffn=self.F_sh, in_dtype=in_dtype, out_dtype=out_dtype, lam=lam,
                                          norm_topk=norm_topk, routed_scale=routed_scale, dedup=dedup,
                                          ffn_impl=ffn_impl, target_reuse=target_reuse)
         self.target_reuse = int(target_reuse)
@@ -276,12 +294,16 @@ class PathMoELayer:
         self.path_tgt = torch.zeros(T, top_k, dtype=torch.int32, device=self.device)
         self.path_w = torch.zeros(T, top_k, dtype=torch.float32, device=self.device)
         self.groups = Groups(max_tokens, top_k, n_experts, self.device)
-        self.y = torch.zeros(T, hidden, dtype=torch.float32, device=self.device)
+        self.out_torch_dtype = torch.bfloat16 if out_dtype == PCOMOE_BF16 else torch.float32
+        self.y = torch.zeros(T, hidden, dtype=self.out_torch_dtype, device=self.device)
         self.in_torch_dtype = torch.bfloat16 if in_dtype == PCOMOE_BF16 else torch.float32
         self._pin_logits = self._pin_h = self._pin_y = None
         self._d_logits = self._d_h = None
 
     def close(self):
+        if getattr(self, "_pipe", None) is not None:
+            self._pipe.close()
+            self._pipe = None
         if self.layer is not None:
             pcomoe_layer_destroy(self.layer)
             self.layer = None
@@ -354,7 +376,7 @@ class PathMoELayer:
             self._pin_logits = torch.empty(cap, self.n, dtype=torch.float32).pin_memory()
             hdt = torch.float32 if h_np.dtype == np.float32 else torch.int16
             self._pin_h = torch.empty(cap, self.H, dtype=hdt).pin_memory()
-            self._pin_y = torch.empty(cap, self.H, dtype=torch.float32).pin_memory()
+            self._pin_y = torch.empty(cap, self.H, dtype=self.out_torch_dtype).pin_memory()
             self._d_logits = torch.empty(cap, self.n, dtype=torch.float32, device=self.device)
             self._d_h = torch.empty(cap, self.H, dtype=hdt, device=self.device)
         self._pin_logits[:T].numpy()[...] = logits_np
@@ -367,7 +389,7 @@ class PathMoELayer:
         y = self.forward(self._d_logits[:T], dh)
         self._pin_y[:T].copy_(y, non_blocking=True)
         torch.cuda.current_stream().synchronize()
-        return self._pin_y[:T].numpy()
+        return self._pin_y[:T].float().numpy()
 
     def capture(self, logits, h, tgt_logits=None):
         """Records one pass of the hot path on fixed device tensors into a CUDA graph and returns it; every
@@ -378,51 +400,82 @@ class PathMoELayer:
             self.forward(logits, h, tgt_logits)
         return g
 
+    def host_pipe(self, slots: int = 2):
+        """The library's host-buffer pipe for this layer (created on first use)."""
+        if getattr(self, "_pipe", None) is None or self._pipe.slots != slots:
+            self._pipe = HostPipe(self, slots)
+        return self._pipe
+
     def stream_from_host(self, pinned_logits, pinned_h, steps: int):
-        """Serving loop over `steps` batches that live in PINNED host memory (torch CPU tensors; `pinned_h` is
-        bf16 or fp32).  Every step copies its inputs host->device, runs the hot path and copies y device->host;
-        the three are put on separate streams with two buffer slots, so the copies of neighbouring steps
-        overlap the kernels.  Returns the pinned y of the last step (synchronised).  Marshalling only."""
+        """Serving loop over `steps` batches that live in pinned host memory (torch CPU tensors), through
+        pcomoe_host_pipe_submit: every step copies its inputs host->device, runs the hot path and copies y
+        device->host, the three overlapped across neighbouring steps inside the library.  Returns the pinned y of
+        the last step (synchronised).  Marshalling only."""
         T = pinned_h.shape[0]
         assert pinned_logits.is_pinned() and pinned_h.is_pinned() and T <= self.max_tokens
-        if getattr(self, "_slots", None) is None or self._slots["T"] < T:
-            mk = lambda *shape, dtype: [torch.empty(*shape, dtype=dtype, device=self.device) for _ in range(2)]
-            self._slots = dict(T=T, logits=mk(T, self.n, dtype=torch.float32), h=mk(T, self.H, dtype=pinned_h.dtype),
-                               y=mk(T, self.H, dtype=torch.float32),
-                               out=[torch.empty(T, self.H, dtype=torch.float32).pin_memory() for _ in range(2)],
-                               s_in=torch.cuda.Stream(self.device), s_out=torch.cuda.Stream(self.device))
-        sl = self._slots
-        main = torch.cuda.current_stream()
-        ev_in = [torch.cuda.Event() for _ in range(2)]
-        ev_done = [torch.cuda.Event() for _ in range(2)]     # kernels of the slot finished (inputs free, y ready)
-        ev_out = [torch.cuda.Event() for _ in range(2)]      # y of the slot copied out (y buffer free)
-        y_keep = self.y
+        pipe = self.host_pipe(2)
+        if getattr(self, "_pin_out", None) is None or self._pin_out[0].shape[0] < T:
+            self._pin_out = [torch.empty(T, self.H, dtype=self.out_torch_dtype).pin_memory() for _ in range(2)]
         for i in range(steps):
-            s = i & 1
-            with torch.cuda.stream(sl["s_in"]):
-                if i >= 2:
-                    sl["s_in"].wait_event(ev_done[s])
-                sl["logits"][s][:T].copy_(pinned_logits[:T], non_blocking=True)
-                sl["h"][s][:T].copy_(pinned_h[:T], non_blocking=True)
-                ev_in[s].record(sl["s_in"])
-            main.wait_event(ev_in[s])
-            if i >= 2:
-                main.wait_event(ev_out[s])
-            self.y = sl["y"][s]
-            self.forward(sl["logits"][s][:T], sl["h"][s][:T])
-            ev_done[s].record(main)
-            with torch.cuda.stream(sl["s_out"]):
-                sl["s_out"].wait_event(ev_done[s])
-                sl["out"][s][:T].copy_(sl["y"][s][:T], non_blocking=True)
-                ev_out[s].record(sl["s_out"])
-        self.y = y_keep
-        last = (steps - 1) & 1
-        ev_out[last].synchronize()
-        main.synchronize()
-        return sl["out"][last][:T]
+            pipe.submit(pinned_logits[:T], pinned_h[:T], self._pin_out[i & 1][:T])
+        st = pipe.wait()
+        if st != PCOMOE_OK:
+            raise PcomoeError(st, "pcomoe_host_pipe_wait")
+        return self._pin_out[(steps - 1) & 1][:T]
 
     def device_status(self) -> int:
         return pcomoe_device_status(self.workspace)
+
+
+class HostPipe:
+    """pcomoe_host_pipe_*: batches in host memory in, y in host memory out.  Marshalling only."""
+
+    def __init__(self, layer: PathMoELayer, slots: int = 2):
+        self.layer, self.slots = layer, slots
+        out = ctypes.c_void_p()
+        _check(load_library().pcomoe_host_pipe_create(layer.layer, layer.max_tokens, slots, _ptr(layer.w_gate),
+                                                      _ptr(layer.w_up), _ptr(layer.w_down), *[_ptr(x) for x in layer.shared],
+                                                      ctypes.byref(out)), "pcomoe_host_pipe_create")
+        self.pipe = out
+
+    @staticmethod
+    def _hptr(a):
+        if a is None:
+            return None
+        if isinstance(a, np.ndarray):
+            assert a.flags.c_contiguous
+            return ctypes.c_void_p(a.ctypes.data)
+        assert a.device.type == "cpu" and a.is_contiguous()
+        return ctypes.c_void_p(a.data_ptr())
+
+    def submit(self, logits, hidden, y_out, tgt_logits=None):
+        """Host arrays (numpy or torch CPU tensors, contiguous; pinned for overlap): logits [T,n] fp32, hidden [T,H]
+        in the layer's input type, y_out [T,H] in its output type.  Returns at once; read y_out after wait()."""
+        T = int(hidden.shape[0])
+        _check(load_library().pcomoe_host_pipe_submit(self.pipe, T, self._hptr(logits), self._hptr(tgt_logits),
+                                                      self._hptr(hidden), self._hptr(y_out)), "pcomoe_host_pipe_submit")
+
+    def wait(self) -> int:
+        return int(load_library().pcomoe_host_pipe_wait(self.pipe))
+
+    def arrays(self, T: int):
+        """Device arrays of the most recent batch as torch tensors (views of the pipe's memory): groups dict, paths."""
+        g = pcomoe_groups()
+        ps, pt, pw = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()
+        _check(load_library().pcomoe_host_pipe_arrays(self.pipe, ctypes.byref(g), ctypes.byref(ps), ctypes.byref(pt),
+                                                      ctypes.byref(pw)), "pcomoe_host_pipe_arrays")
+        return g, ps, pt, pw
+
+    def close(self):
+        if self.pipe is not None:
+            load_library().pcomoe_host_pipe_destroy(self.pipe)
+            self.pipe = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class PathMoEStack:

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "pcomoe.h"
 
 namespace pcomoe {
@@ -49,6 +51,7 @@ struct WsLayout {
   size_t u_sh;         // in_dtype [Tpad, F_sh]      shared-expert intermediates
   size_t h_gath;       // bf16 [mt_max*128, H]       rows of h in padded stage-1 order (tensor-core path)
   size_t path_wgt;     // fp32 [T*K]                 copy of the path weights (projection-side reuse only)
+  size_t y_acc;        // fp32 [T, H]                fp32 accumulator of y when the layer's output type is bf16
   size_t total;
   int32_t nb_max;      // blocks of the grouping kernels at max_tokens
   int32_t mt_max;      // upper bound of m-tiles per stage
@@ -74,6 +77,7 @@ namespace pcomoe {
 
 WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens);
 void count_launch(int n = 1);
+uint64_t wait_limit_ns();            // limit of every bounded device-side wait (pcomoe_set_wait_limit_us)
 
 inline size_t dtype_size(int dt) { return dt == PCOMOE_BF16 ? 2 : 4; }
 
@@ -92,6 +96,19 @@ inline int group_chunk_for(const pcomoe_layer *L, int32_t T) {
   while (chunk > 32 && (int64_t)T / chunk < 2 * (int64_t)L->sm_count) chunk >>= 1;
   return chunk;
 }
+
+// Kernel attributes (cudaFuncSetAttribute) belong to a device: a once-flag per device ordinal.  first_use()
+// is true until done() has been called for that device; setting the attributes twice is harmless, so a race
+// between two threads only repeats the calls.  Devices beyond the table set their attributes on every call.
+struct PerDeviceOnce {
+  std::atomic<uint64_t> mask{0};
+  bool first_use(int device) const {
+    return device < 0 || device >= 64 || !((mask.load(std::memory_order_acquire) >> device) & 1u);
+  }
+  void done(int device) {
+    if (device >= 0 && device < 64) mask.fetch_or(uint64_t(1) << device, std::memory_order_release);
+  }
+};
 
 #define PCOMOE_CUDA_TRY(expr)                          \
   do {                                                 \
@@ -132,6 +149,8 @@ pcomoe_status launch_route(const pcomoe_layer *L, int32_t T, const float *z, con
 pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, const void *w_router,
                             const void *lora_a, const float *lora_b, int32_t r, float scale, float *logits,
                             int32_t *status, cudaStream_t st);
+pcomoe_status launch_cast_y(const pcomoe_layer *L, int32_t T, const float *y_acc, void *y_out, cudaStream_t st);
+pcomoe_status launch_wait_probe(int32_t *status_word, cudaStream_t st);
 pcomoe_status launch_residual_cast(const pcomoe_layer *L, int32_t T, const void *h_in, const float *y, void *h_out,
                                    cudaStream_t st);
 pcomoe_status launch_groups(const pcomoe_layer *L, int32_t T, const int32_t *src, const int32_t *tgt,

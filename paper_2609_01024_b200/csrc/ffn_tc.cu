@@ -67,6 +67,7 @@ struct TcParams {
   float4 *zero_ptr;            // stage 1 only: buffer the epilogue warps clear before their first tile
   int64_t zero_vec4;           //               (y, so that stage 2 can accumulate into it); 0: nothing
   DevPlan *plan;
+  uint64_t wait_ns;            // limit of every mbarrier wait
 };
 
 // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256
@@ -431,7 +432,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
         const int a_row0 = t.prow0;
         const int b_row = t.g * S.b_group_rows + t.n_idx * (STAGE == 1 ? 128 : 256);
         for (int kb = 0; kb < S.kb; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_ns)) { alive = false; break; }
           const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + A_BYTES;
           mbar_arrive_expect_tx(full_bar(stage), STAGE_BYTES);
           tma_load_2d(sa, mA, kb * BK, a_row0, full_bar(stage));
@@ -455,11 +456,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
       for (int tile = blockIdx.x; tile < total && alive; tile += gridDim.x) {
         const TileInfo t = walk.at(tile);
         const int nkb = p.seg[t.seg].kb;
-        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
+        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_ns)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
         for (int kb = 0; kb < nkb; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_ns)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = ring + stage * STAGE_BYTES, sb = sa + A_BYTES;
           const uint64_t da = umma_desc(sa), db = umma_desc(sb);
@@ -495,7 +496,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
       const DstList dl{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0), s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
                        s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)};
       const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r, dl);
-      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
+      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.wait_ns)) break;
       tc_fence_after();
       epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
                            s_epi + (warp - 2) * 32 * kEpiStride, dl);
@@ -509,10 +510,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
   tc_fence_before();
   __syncthreads();
   if (s_abort) {
-    if (threadIdx.x == 0) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_TIMEOUT);
-    // let copies and MMAs already issued finish before shared memory and TMEM are given back
-    const uint64_t t0 = global_ns();
-    for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
+    timeout_record_and_drain(&p.plan->status);
     __syncthreads();
   }
   if (warp == 1) {
@@ -728,7 +726,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
           b_row = t.g * S.b_group_rows + t.n_idx * 256 + (int)rank * 128;
         }
         for (int kb = 0; kb < S.kb; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_ns)) { alive = false; break; }
           const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
           const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
@@ -748,11 +746,11 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
       for (int tile = pair_id; tile < total && alive; tile += n_pairs) {
         const TileInfo t = walk.at(tile, 0);
         const int nkb = p.seg[t.seg].kb;
-        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
+        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_ns)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
         for (int kb = 0; kb < nkb; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_ns)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
           const uint64_t da = umma_desc(sa), db = umma_desc(sb);
@@ -787,7 +785,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
       const DstList dl{s_dl_dst + (STAGE == 1 ? (warp - 2) * kDstList : 0), s_dl_row + (STAGE == 1 ? (warp - 2) * kDstList : 0),
                        s_dl_w + ((STAGE == 1 && MERGE) ? (warp - 2) * kDstList : 0)};
       const RowCtx c = prepare_row<STAGE, MERGE>(p, S, t, r, dl);
-      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag)) break;
+      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.wait_ns)) break;
       tc_fence_after();
       epilogue_tile<STAGE, MERGE>(p, S, t, c, tmem_base + acc * ACC_COLS + ((uint32_t)(quarter * 32) << 16),
                            s_epi + (warp - 2) * 32 * kEpiStride, dl);
@@ -800,11 +798,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
   // ---------------- teardown ----------------
   tc_fence_before();
   __syncthreads();
-  if (s_abort) {
-    if (threadIdx.x == 0) atomicCAS(&p.plan->status, 0, PCOMOE_ERR_TIMEOUT);
-    const uint64_t t0 = global_ns();
-    for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
-  }
+  if (s_abort) timeout_record_and_drain(&p.plan->status);
   cluster_sync_all();                 // no signal may reach a CTA that has already exited
   if (warp == 1) {
     __syncwarp();
@@ -879,18 +873,19 @@ pcomoe_status launch_shared_stage1_side(const pcomoe_layer *L, int32_t T, const 
   if (!L->tc_ok || Fsh <= 0) return PCOMOE_ERR_UNSUPPORTED;
   DevPlan *plan = reinterpret_cast<DevPlan *>(ws + lay.plan);
   __nv_bfloat16 *Ush = reinterpret_cast<__nv_bfloat16 *>(ws + lay.u_sh);
-  static bool attr_done = false;
+  static PerDeviceOnce attr_once;
   auto kern = grouped_gemm_pair_kernel<1, false, kSideStages>;
-  if (!attr_done) {
+  if (attr_once.first_use(L->device)) {
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemSide));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
-    attr_done = true;
+    attr_once.done(L->device);
   }
   CUtensorMap mA, mB, mC;
   // tokens [0, rows) only: the rest of the shared expert's stage 1 rides in the main stage-1 launch
   if (!(make_map(&mA, h, (uint64_t)rows, H, kTileM) && make_map(&mB, sg, Fsh, H, 128) && make_map(&mC, su, Fsh, H, 128)))
     return PCOMOE_ERR_CUDA;
   TcParams p{};
+  p.wait_ns = wait_limit_ns();
   p.K = c.top_k; p.T = T; p.y = nullptr; p.ldy = H;
   // only the status word of the plan is touched by the kernel: point it at the router's word
   p.plan = reinterpret_cast<DevPlan *>(reinterpret_cast<char *>(plan) + offsetof(DevPlan, status_router));
@@ -923,15 +918,15 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   const size_t pad_rows = (size_t)lay.mt_max * kTileM;
   if (Fsh == 0) stages &= ~(kStage1Shared | kStage2Shared);
 
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;
+  if (attr_once.first_use(L->device)) {
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
-    attr_done = true;
+    attr_once.done(L->device);
   }
   const bool pair = use_cta_pairs(L, T);
   const int grid = pair ? (L->sm_count & ~1) : L->sm_count;
@@ -955,6 +950,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   if (stages & (kStage1Routed | kStage1Shared)) {
     CUtensorMap mA[2], mB[2], mC[2];
     TcParams p{};
+    p.wait_ns = wait_limit_ns();
     p.K = c.top_k; p.T = T; p.plan = plan; p.y = y; p.ldy = H;
     int ns = 0;
     bool ok = true;
@@ -999,6 +995,7 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   if (stages & (kStage2Routed | kStage2Shared)) {
     CUtensorMap mA[2], mB[2];
     TcParams p{};
+    p.wait_ns = wait_limit_ns();
     p.K = c.top_k; p.T = T; p.plan = plan; p.y = y; p.ldy = H;
     int ns = 0;
     bool ok = true;

@@ -17,6 +17,9 @@ namespace pcomoe {
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+static std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};   // 2 s
+uint64_t wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
+
 static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
@@ -49,6 +52,7 @@ WsLayout ws_layout(const pcomoe_layer *L, int32_t max_tokens) {
   w.u_sh = take(es * (size_t)w.t_pad * c.shared_ffn);
   if (L->tc_ok) w.h_gath = take(es * (size_t)w.mt_max * kTileM * c.hidden);
   if (c.target_reuse) w.path_wgt = take(sizeof(float) * (size_t)Pm);
+  if (c.out_dtype == PCOMOE_BF16) w.y_acc = take(sizeof(float) * (size_t)Tm * c.hidden);
   w.total = off;
   return w;
 }
@@ -76,7 +80,7 @@ pcomoe_status pcomoe_layer_create(const pcomoe_config *cfg, const uint8_t *h_mas
     return PCOMOE_ERR_INVALID_ARG;
   if (K > n || K > kMaxTopK) return PCOMOE_ERR_SHAPE;
   if (n > kMaxExperts) return PCOMOE_ERR_UNSUPPORTED;
-  if (cfg->out_dtype != PCOMOE_FP32) return PCOMOE_ERR_UNSUPPORTED;
+  if (cfg->out_dtype != PCOMOE_FP32 && cfg->out_dtype != PCOMOE_BF16) return PCOMOE_ERR_INVALID_ARG;
   if (cfg->hidden % 8 || cfg->ffn % 8 || cfg->shared_ffn % 8) return PCOMOE_ERR_UNSUPPORTED;
   for (int i = 0; i < n; ++i)
     if (!h_mask[(size_t)i * n + i]) return PCOMOE_ERR_INVALID_ARG;  // m_ii = 1 (Sec. 4.2)
@@ -272,11 +276,18 @@ pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *L, int32_t T, const 
   if (s != PCOMOE_OK) return s;
   const bool tc = L->cfg.ffn_impl >= PCOMOE_FFN_TCGEN05 ||
                   (L->cfg.ffn_impl == PCOMOE_FFN_AUTO && L->tc_ok);
+  // a bf16 output is accumulated in fp32 in the workspace and rounded once, after the last addition
+  const bool y_bf16 = L->cfg.out_dtype == PCOMOE_BF16;
+  float *y_acc = y_bf16 ? reinterpret_cast<float *>((char *)d_workspace + lay.y_acc) : (float *)d_y;
   if (tc)
-    return launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
-                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
-  return launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
-                         groups, (float *)d_y, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
+    s = launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
+                      groups, y_acc, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
+  else
+    s = launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down,
+                        groups, y_acc, (char *)d_workspace, lay, (cudaStream_t)stream, stages);
+  if (s == PCOMOE_OK && y_bf16 && (stages & (kStage2Routed | kStage2Shared)))
+    s = launch_cast_y(L, T, y_acc, d_y, (cudaStream_t)stream);
+  return s;
 }
 
 pcomoe_status pcomoe_layer_forward(const pcomoe_layer *L, int32_t T, const float *d_logits,
@@ -323,18 +334,21 @@ pcomoe_status pcomoe_layer_forward(const pcomoe_layer *L, int32_t T, const float
       return s;
     }
   }
+  const bool y_bf16 = L->cfg.out_dtype == PCOMOE_BF16;
+  float *y_acc = y_bf16 ? reinterpret_cast<float *>((char *)d_workspace + lay.y_acc) : (float *)d_y;
   s = launch_route(L, T, d_logits, d_tgt_logits ? d_tgt_logits : d_logits, d_path_src, d_path_tgt, d_path_w, st);
   if (s == PCOMOE_OK)
     s = launch_groups(L, T, d_path_src, d_path_tgt, d_path_w, groups, (char *)d_workspace, lay, st);
   if (s == PCOMOE_OK) {
     if (tc)
       s = launch_ffn_tc(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down, groups,
-                        (float *)d_y, (char *)d_workspace, lay, st,
+                        y_acc, (char *)d_workspace, lay, st,
                         !overlap ? 15 : side_rows < T ? 15 : (kStage1Routed | kStage2Routed | kStage2Shared),
                         overlap ? L->ev_join : nullptr, side_rows);
     else
       s = launch_ffn_simt(L, T, d_h, d_w_gate, d_w_up, d_w_down, d_wsh_gate, d_wsh_up, d_wsh_down, groups,
-                          (float *)d_y, (char *)d_workspace, lay, st, 15);
+                          y_acc, (char *)d_workspace, lay, st, 15);
+    if (s == PCOMOE_OK && y_bf16) s = launch_cast_y(L, T, y_acc, d_y, st);
   } else if (overlap) {
     cudaStreamWaitEvent(st, L->ev_join, 0);
   }
@@ -382,6 +396,20 @@ pcomoe_status pcomoe_device_status(const void *d_workspace, void *stream) {
   }
   if (st < 0 || st > PCOMOE_ERR_INDEX) return PCOMOE_ERR_CUDA;
   return (pcomoe_status)st;
+}
+
+pcomoe_status pcomoe_set_wait_limit_us(uint32_t limit_us) {
+  if (limit_us == 0) limit_us = 2000000u;
+  if (limit_us > 60000000u) return PCOMOE_ERR_INVALID_ARG;
+  g_wait_limit_ns.store((uint64_t)limit_us * 1000ull, std::memory_order_relaxed);
+  return PCOMOE_OK;
+}
+
+pcomoe_status pcomoe_selftest_wait_timeout(void *d_workspace, void *stream) {
+  if (!d_workspace) return PCOMOE_ERR_WORKSPACE;
+  if (((uintptr_t)d_workspace) & 255) return PCOMOE_ERR_WORKSPACE;
+  DevPlan *plan = reinterpret_cast<DevPlan *>(d_workspace);
+  return launch_wait_probe(&plan->status, (cudaStream_t)stream);
 }
 
 int64_t pcomoe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -26,11 +26,16 @@ struct RouteParams {
   int32_t cache_scores;      // pass 1 keeps the scores in shared memory for pass 2
 };
 
+// A NaN or infinite score takes the path out of the token's active set: it becomes -inf, which ranks after every
+// finite score and is never written out as a selection (a token with fewer than K finite scores gets -1 ids and
+// weight 0 in the ranks it cannot fill; the grouping step skips such paths and reports PCOMOE_ERR_INDEX).
+__device__ __forceinline__ float drop_non_finite(float s) { return fabsf(s) <= FLT_MAX ? s : -INFINITY; }
+
 __device__ __forceinline__ float path_score(const ActiveEntry e, const float *zs, const float *us,
                                             float lambda) {
   float a = __fadd_rn(zs[e.src], e.bias);
   float b = __fmul_rn(lambda, us[e.tgt]);
-  return __fadd_rn(__fadd_rn(a, b), 0.0f);  // the last add turns -0 into +0
+  return drop_non_finite(__fadd_rn(__fadd_rn(a, b), 0.0f));  // the last add turns -0 into +0
 }
 
 // true when (s1,a1) ranks before (s2,a2)
@@ -49,7 +54,7 @@ __device__ __noinline__ void topk_by_lists(const RouteParams &p, const ActiveEnt
   int la[KMAX];
 #pragma unroll
   for (int i = 0; i < KMAX; ++i) {
-    ls[i] = -FLT_MAX;
+    ls[i] = -INFINITY;
     la[i] = 0x7fffffff;
   }
   for (int a = lane; a < p.A; a += 32) {
@@ -84,7 +89,7 @@ __device__ __noinline__ void topk_by_lists(const RouteParams &p, const ActiveEnt
         ls[i] = ls[i + 1];
         la[i] = la[i + 1];
       }
-      ls[KMAX - 1] = -FLT_MAX;
+      ls[KMAX - 1] = -INFINITY;
       la[KMAX - 1] = 0x7fffffff;
     }
     if (lane == k) {
@@ -140,7 +145,7 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
     // so every path of the TopK scores >= tau, and usually only a handful of paths do.  Those candidates
     // (ties with tau included) are compacted one per lane and ranked exactly; when more than 32 qualify
     // (heavy ties) the token falls back to the per-lane lists, which give the same selection.
-    float m = -FLT_MAX;
+    float m = -INFINITY;
     for (int a = lane; a < p.A; a += 32) {
       const float s = path_score(tab[a], zs, us, p.lambda);
       if (cache) cache[a] = s;
@@ -150,7 +155,7 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
     for (int k = 0; k < p.K; ++k) {
       tau = warp_max(m);
       const unsigned hit = __ballot_sync(0xffffffffu, m == tau);
-      if (lane == __ffs(hit) - 1) m = -FLT_MAX;
+      if (lane == __ffs(hit) - 1) m = -INFINITY;
     }
     int cnt = 0;
     for (int i = 0; i < rounds; ++i) {
@@ -173,10 +178,10 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
     }
     __syncwarp();
 
-    float my_s = -FLT_MAX;
+    float my_s = -INFINITY;
     int my_a = 0;
     if (cnt <= 32) {
-      float cs = lane < cnt ? cand_s[lane] : -FLT_MAX;
+      float cs = lane < cnt ? cand_s[lane] : -INFINITY;
       int ca = lane < cnt ? cand_a[lane] : 0x7fffffff;
       for (int k = 0; k < p.K; ++k) {
         float bs = cs;
@@ -191,7 +196,7 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
           }
         }
         if (ca == ba) {
-          cs = -FLT_MAX;
+          cs = -INFINITY;
           ca = 0x7fffffff;
         }
         if (lane == k) {
@@ -204,7 +209,8 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
     }
 
     const float s0 = __shfl_sync(0xffffffffu, my_s, 0);
-    float e = lane < p.K ? expf(my_s - s0) : 0.0f;
+    const bool live = lane < p.K && my_s > -INFINITY && (unsigned)my_a < (unsigned)p.A;
+    float e = live ? expf(my_s - s0) : 0.0f;
     float den;
     if (p.norm_topk) {
       den = e;
@@ -215,11 +221,17 @@ __global__ void __launch_bounds__(256) route_kernel(const RouteParams p) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
     if (lane < p.K) {
-      const ActiveEntry en = tab[my_a];
       const size_t o = (size_t)t * p.K + lane;
-      p.src[o] = en.src;
-      p.tgt[o] = en.tgt;
-      p.w[o] = e / den * p.scale;
+      if (live) {
+        const ActiveEntry en = tab[my_a];
+        p.src[o] = en.src;
+        p.tgt[o] = en.tgt;
+        p.w[o] = e / den * p.scale;
+      } else {   // no finite score left for this rank
+        p.src[o] = -1;
+        p.tgt[o] = -1;
+        p.w[o] = 0.0f;
+      }
     }
   }
 }
@@ -279,7 +291,7 @@ __global__ void __launch_bounds__(256) route_fast_kernel(const RouteParams p) {
       const uint4 e = st4[a];
       const float zi = *reinterpret_cast<const float *>(rb + e.x);
       const float uj = *reinterpret_cast<const float *>(rb + e.y);
-      const float s = __fadd_rn(__fadd_rn(zi, __uint_as_float(e.z)), uj);
+      const float s = drop_non_finite(__fadd_rn(__fadd_rn(zi, __uint_as_float(e.z)), uj));
       cache[a] = s;
       m = fmaxf(m, s);
     }
@@ -312,7 +324,7 @@ __global__ void __launch_bounds__(256) route_fast_kernel(const RouteParams p) {
     __syncwarp();
     const int cnt = *cand_n;
 
-    float my_s = -FLT_MAX;
+    float my_s = -INFINITY;
     int my_a = 0;
     if (cnt <= 32) {
       // rank by counting: the position of a candidate is the number of candidates that rank before it
@@ -341,7 +353,8 @@ __global__ void __launch_bounds__(256) route_fast_kernel(const RouteParams p) {
     }
 
     const float s0 = __shfl_sync(0xffffffffu, my_s, 0);
-    float e = lane < p.K ? expf(my_s - s0) : 0.0f;
+    const bool live = lane < p.K && my_s > -INFINITY && (unsigned)my_a < (unsigned)A;
+    float e = live ? expf(my_s - s0) : 0.0f;
     float den;
     if (p.norm_topk) {
       den = e;
@@ -352,11 +365,17 @@ __global__ void __launch_bounds__(256) route_fast_kernel(const RouteParams p) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
     if (lane < p.K) {
-      const ActiveEntry en = p.table[my_a];
       const size_t o = (size_t)t * p.K + lane;
-      p.src[o] = en.src;
-      p.tgt[o] = en.tgt;
-      p.w[o] = e / den * p.scale;
+      if (live) {
+        const ActiveEntry en = p.table[my_a];
+        p.src[o] = en.src;
+        p.tgt[o] = en.tgt;
+        p.w[o] = e / den * p.scale;
+      } else {   // no finite score left for this rank
+        p.src[o] = -1;
+        p.tgt[o] = -1;
+        p.w[o] = 0.0f;
+      }
     }
   }
 }

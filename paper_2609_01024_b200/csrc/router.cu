@@ -35,6 +35,7 @@ struct RouterParams {
   uint32_t stage_bytes;   // kRA + n_mma * 128
   uint32_t idesc, tmem_cols;
   float scale;
+  uint64_t wait_ns;       // limit of every mbarrier wait
 };
 
 __device__ __forceinline__ void umma_bf16_n(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
@@ -123,7 +124,7 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       int stage = 0;
       uint32_t phase = 0;
       for (int kb = kb_lo; kb < kb_hi; ++kb) {
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) break;
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_ns)) break;
         const uint32_t sa = ring + stage * p.stage_bytes, sb = sa + kRA;
         mbar_arrive_expect_tx(full_bar(stage), stage_tx);
         tma_load_2d(sa, &tmH, kb * BK, row0, full_bar(stage));
@@ -139,7 +140,7 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
       uint32_t phase = 0;
       bool alive = true;
       for (int kb = kb_lo; kb < kb_hi; ++kb) {
-        if (!mbar_wait(full_bar(stage), phase, abort_flag)) { alive = false; break; }
+        if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_ns)) { alive = false; break; }
         tc_fence_after();
         const uint32_t sa = ring + stage * p.stage_bytes, sb = sa + kRA;
         const uint64_t da = umma_desc(sa), db = umma_desc(sb);
@@ -154,7 +155,7 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
     __syncwarp();
   }
   // every thread waits for the accumulator: the ring is free after that and becomes the turn-around buffer
-  const bool done = mbar_wait(acc_bar, 0, abort_flag);
+  const bool done = mbar_wait(acc_bar, 0, abort_flag, p.wait_ns);
   tc_fence_after();
   __syncthreads();
   float *turn = reinterpret_cast<float *>(ring_ptr);          // [128][n_mma + 1] fp32: this CTA's partial sums
@@ -220,9 +221,7 @@ router_gemm_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constan
   if (p.split > 1) cluster_barrier();                         // peers may still be reading this CTA's sums
   // ---------------- teardown ----------------
   if (s_abort) {
-    if (threadIdx.x == 0 && p.status) atomicCAS(p.status, 0, PCOMOE_ERR_TIMEOUT);
-    const uint64_t t0 = global_ns();
-    for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
+    if (p.status) timeout_record_and_drain(p.status);
     __syncthreads();
   }
   if (warp == 1) {
@@ -294,6 +293,7 @@ pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, con
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)n_mma >> 3) << 17) | ((128u >> 4) << 24);
     p.tmem_cols = n_mma <= 32 ? 32u : n_mma <= 64 ? 64u : n_mma <= 128 ? 128u : 256u;
     p.scale = scale;
+    p.wait_ns = wait_limit_ns();
     p.stage_bytes = kRA + (uint32_t)n_mma * (BK * 2);
     p.stages = (int)((kRSmem - 1024) / p.stage_bytes);
     if (p.stages > kRMaxStages) p.stages = kRMaxStages;
@@ -303,10 +303,10 @@ pcomoe_status launch_router(const pcomoe_layer *L, int32_t T, const void *h, con
     int split = 1;
     while (split < 8 && tiles * split * 2 <= L->sm_count && p.kb >= 4 * split && n_mma <= 128) split *= 2;
     p.split = split;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    if (attr_once.first_use(L->device)) {
       PCOMOE_CUDA_TRY(cudaFuncSetAttribute(router_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRSmem));
-      attr_done = true;
+      attr_once.done(L->device);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles * split);

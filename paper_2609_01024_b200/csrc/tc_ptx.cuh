@@ -10,7 +10,6 @@ namespace pcomoe {
 namespace {
 
 constexpr int BK = 64;                      // k-block: 64 bf16 = one 128-byte swizzle row
-constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -43,17 +42,27 @@ __device__ __forceinline__ uint64_t global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait.  Returns false when the CTA is giving up (this or another role timed out).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// Bounded wait: gives up after `limit_ns` (the library-wide limit, see wait_limit_ns(); the kernels carry it in
+// their parameters).  Returns false when the CTA is giving up (this or another role timed out).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t it = 1; it < (1u << 24); ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitLimitNs) break;
+    if (global_ns() - t0 > limit_ns) break;
   }
   *abort_flag = 1;
   return false;
+}
+
+// What a CTA does once one of its waits has run out: record the timeout in the status word, then give the
+// copies and MMAs already issued time to finish before shared memory and TMEM are given back.  All threads
+// of the CTA call it.
+__device__ __forceinline__ void timeout_record_and_drain(int32_t *status_word) {
+  if (threadIdx.x == 0) atomicCAS(status_word, 0, (int32_t)PCOMOE_ERR_TIMEOUT);
+  const uint64_t t0 = global_ns();
+  for (int it = 0; it < (1 << 22) && global_ns() - t0 < 200000ull; ++it) __nanosleep(256);
 }
 
 // L2 eviction policy of the weight loads in the one-CTA kernel: it serves decode-sized batches, where a weight

@@ -9,7 +9,8 @@ GROUP_KEYS = ("s1_offsets", "s1_token", "path_s1row", "s2_offsets", "s2_path", "
 
 
 def make_gpu_layer(cfg, L, *, mask=None, bias=None, lam=None, norm_topk=1, routed_scale=1.0, dedup=1,
-                   ffn_impl=B.PCOMOE_FFN_AUTO, max_tokens=None, with_weights=True, target_reuse=0):
+                   ffn_impl=B.PCOMOE_FFN_AUTO, max_tokens=None, with_weights=True, target_reuse=0,
+                   out_dtype=B.PCOMOE_FP32):
     dev = "cuda:0"
     dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
     if with_weights:
@@ -23,7 +24,7 @@ def make_gpu_layer(cfg, L, *, mask=None, bias=None, lam=None, norm_topk=1, route
                           w_gate=wg, w_up=wu, w_down=wd, shared=shared if (with_weights and cfg.F_sh) else None,
                           max_tokens=cfg.T if max_tokens is None else max_tokens, in_dtype=dt,
                           lam=cfg.lam if lam is None else lam, norm_topk=norm_topk, routed_scale=routed_scale,
-                          dedup=dedup, ffn_impl=ffn_impl, target_reuse=target_reuse, device=dev)
+                          dedup=dedup, ffn_impl=ffn_impl, target_reuse=target_reuse, out_dtype=out_dtype, device=dev)
 
 
 def route_on_gpu(layer, logits, tgt_logits=None):

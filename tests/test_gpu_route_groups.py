@@ -93,6 +93,49 @@ def test_adversarial_routing_cases(G, oracle, case):
         assert np.all(src[:, 0] == 4)
 
 
+@pytest.mark.parametrize("shape", [(9, 3, 0.4), (60, 4, 0.3), (6, 6, 1.0), (40, 2, 1.0)])
+@pytest.mark.parametrize("norm_topk", [1, 0])
+def test_non_finite_logits_never_fault(G, oracle, shape, norm_topk):
+    """-inf (a router that masks experts), +inf and NaN logits: the selection is the oracle's, ranks without a
+    finite score carry -1 ids and weight 0, and the grouping step skips them and raises its status word."""
+    n, K, p = shape
+    rng = np.random.default_rng(n * 100 + K)
+    T = 257
+    z = rng.standard_normal((T, n)).astype(np.float32)
+    M = (rng.random((n, n)) < p).astype(np.uint8); np.fill_diagonal(M, 1)
+    Bm = (-1.0 + 0.25 * rng.standard_normal((n, n))).astype(np.float32); np.fill_diagonal(Bm, 0.0)
+    z[:, 1] = -np.inf                                   # one expert masked for every token
+    z[5] = np.nan                                        # an all-NaN row
+    z[6, 0] = np.nan                                     # a row with a single NaN
+    z[7] = -np.inf                                       # every expert masked
+    z[8, : n - 1] = -np.inf                              # one expert left: fewer than K finite scores when K > 1
+    z[9, 2] = np.inf                                     # +inf
+    z[10:40][rng.random((30, n)) < 0.7] = -np.inf       # many masked experts, different per token
+    z[40:60][rng.random((20, n)) < 0.3] = np.nan
+    cfg = wl.small_case(1, T=T, H=64, F=64, n=n, K=K, lam=0.5)
+    L = wl.make_layer(cfg, with_weights=False)
+    layer = G.make_gpu_layer(cfg, L, with_weights=False, mask=M, bias=Bm, lam=0.5, norm_topk=norm_topk)
+    src, tgt, w = G.route_on_gpu(layer, z)
+    rs, rt, rw = oracle.route(z, M, Bm, 0.5, K, norm_topk=norm_topk)
+    assert np.array_equal(src, rs) and np.array_equal(tgt, rt)
+    assert np.all(np.isfinite(w))
+    np.testing.assert_allclose(w, rw, rtol=0, atol=1e-6)
+    assert (rs[5] == -1).all() and (rs[7] == -1).all() and (w[rs < 0] == 0).all()
+    g, st = G.groups_on_gpu(layer, src, tgt, w)
+    assert st == 7                                       # PCOMOE_ERR_INDEX: some paths were skipped
+    ref = oracle.groups(src, tgt, w, n)
+    assert g["R1"] == ref["R1"]
+    P = int(ref["s2_offsets"][-1])
+    assert P == int((rs >= 0).sum())
+    for k in ("s1_offsets", "s2_offsets"):
+        assert np.array_equal(g[k], ref[k]), k
+    assert np.array_equal(np.asarray(g["s1_token"])[:ref["R1"]], ref["s1_token"][:ref["R1"]])
+    for k in ("s2_path", "s2_s1row", "s2_token", "s2_w"):
+        assert np.array_equal(np.asarray(g[k])[:P], ref[k][:P]), k
+    live = rs >= 0
+    assert np.array_equal(np.asarray(g["path_s1row"]).reshape(T, K)[live], ref["path_s1row"][live])
+
+
 def test_empty_batch_and_bad_indices(G, oracle):
     cfg = wl.small_case(2, T=40, H=64, F=64, n=6, K=2)
     L = wl.make_layer(cfg, with_weights=False)

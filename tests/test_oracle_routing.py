@@ -164,3 +164,30 @@ def test_unnormalised_mass_is_at_most_one(oracle):
     _, _, w0 = oracle.route(z, M, B, 0.5, K, norm_topk=0)
     assert np.all(w0.sum(-1) < 1.0)
     np.testing.assert_allclose(w0 / w0.sum(-1, keepdims=True), w1, atol=1e-6)
+
+
+def test_non_finite_scores_leave_the_active_set(oracle):
+    """Reading for inputs the paper does not consider: a path with a NaN or infinite score is not eligible
+    for that token; ranks that cannot be filled carry -1 ids and weight 0.  Worked by hand."""
+    n, K, lam = 3, 2, 0.5
+    M = np.ones((n, n), np.uint8)
+    B = np.zeros((n, n), np.float32)
+    inf, nan = np.float32(np.inf), np.float32(np.nan)
+    z = np.array([[1.0, -inf, 0.0],      # expert 1 masked by the router: paths through it drop out
+                  [nan, nan, nan],       # nothing is eligible
+                  [-inf, -inf, 2.0],     # only path (2,2) is finite
+                  [inf, 0.0, 0.0]], np.float32)   # +inf is dropped like any other non-finite score
+    src, tgt, w = oracle.route(z, M, B, lam, K)
+    # token 0: finite scores (0,0)=1.5, (0,2)=1.0, (2,0)=0.5, (2,2)=0
+    assert src[0].tolist() == [0, 0] and tgt[0].tolist() == [0, 2]
+    np.testing.assert_allclose(w[0], [1 / (1 + np.exp(-0.5)), 1 - 1 / (1 + np.exp(-0.5))], atol=1e-7)
+    assert src[1].tolist() == [-1, -1] and tgt[1].tolist() == [-1, -1] and w[1].tolist() == [0.0, 0.0]
+    assert src[2].tolist() == [2, -1] and tgt[2].tolist() == [2, -1] and w[2].tolist() == [1.0, 0.0]
+    # token 3: every path that touches expert 0 is +inf; the finite ones are (1,1),(1,2),(2,1),(2,2), all 0
+    assert src[3].tolist() == [1, 1] and tgt[3].tolist() == [1, 2]
+    np.testing.assert_allclose(w[3], [0.5, 0.5], atol=1e-7)
+    # rows without a non-finite value are decided exactly as before
+    zz = np.random.default_rng(0).standard_normal((20, n)).astype(np.float32)
+    a = oracle.route(zz, M, B, lam, K)
+    flat = a[0].astype(np.int64) * n + a[1]
+    assert np.array_equal(flat, _py_route(zz, zz, M, B, lam, K))
