@@ -31,9 +31,6 @@ from paper_2609_01024_b200 import workloads as wl  # noqa: E402
 
 METRIC = "path_moe_layer_tokens_per_s"
 UNIT = "tokens/s"
-# DRAM bytes (dram__bytes_read + dram__bytes_write) of ONE launch of the dominant kernel (stage-1 grouped GEMM) on
-# the benchmark layers, from the ncu capture summarised in profiles/kernels_per_config.md
-NCU_TRAFFIC_STAGE1 = {2: 2321.7e6, 3: 1119.4e6, 4: 1257.2e6, 5: 1890.9e6}   # routed groups only (the launch the stage-1 time is taken from)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -46,6 +43,15 @@ def peaks():
     d = dict(FALLBACK_PEAKS)
     d["source"] = "fallback"
     return d
+
+
+def ncu_traffic_stage1(config_index):
+    """DRAM bytes (read + write) of one launch of the dominant kernel from the committed profiler summary, or None."""
+    p = os.path.join(ROOT, "profiles", "stage1_dram_traffic.json")
+    try:
+        return json.load(open(p))["bytes_per_launch"].get(str(config_index))
+    except Exception:
+        return None
 
 
 class ClockSampler:
@@ -107,7 +113,11 @@ class ClockSampler:
             try:
                 mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
                 r = int(get_reasons(self.handle)) if get_reasons else 0
-                self.rows.append((time.time(), mhz, self.max_mhz, {name for name, b in bits if r & b}))
+                try:
+                    pw = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                except Exception:
+                    pw = None
+                self.rows.append((time.time(), mhz, self.max_mhz, {name for name, b in bits if r & b}, pw))
             except Exception:
                 pass
             time.sleep(0.004)
@@ -118,7 +128,11 @@ class ClockSampler:
             try:
                 rs = {name for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
                                                "sw_power_cap"), f[4:8]) if v == "Active"}
-                self.rows.append((time.time(), float(f[1]), float(f[2]), rs))
+                try:
+                    pw = float(f[3])
+                except Exception:
+                    pw = None
+                self.rows.append((time.time(), float(f[1]), float(f[2]), rs, pw))
             except Exception:
                 continue
 
@@ -131,13 +145,27 @@ class ClockSampler:
         if self.proc is not None:
             time.sleep(0.05)
             self.proc.terminate()
-        sm, mx, reasons = [], [], set()
-        for ts, mhz, mmax, rs in list(self.rows):
+        return self.window(t0, t1)
+
+    def window(self, t0=None, t1=None):
+        """Summary of the samples taken in [t0, t1].  A sample counts as "under load" when the board drew more
+        than 400 W; the driver's clock reading trails the hardware by tens of milliseconds, so in a timed region
+        that short the clocks shown can still be the idle ones (the power-cap reason is the better witness)."""
+        sm, mx, reasons, pw, sm_load = [], [], set(), [], []
+        for ts, mhz, mmax, rs, p in list(self.rows):
             if t0 is not None and not (t0 <= ts <= t1 + 0.03):
                 continue
             sm.append(mhz); mx.append(mmax); reasons |= rs
+            if p is not None:
+                pw.append(p)
+                if p > 400.0:
+                    sm_load.append(mhz)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm),
+                "samples_under_load": len(sm_load),
+                "sm_mhz_under_load": statistics.median(sm_load) if sm_load else None,
+                "power_w_max": max(pw) if pw else None,
+                "note": "driver clock readings lag a region of tens of ms; sw_power_cap during a dense GEMM is normal",
                 "source": "+".join(x for x, on in (("nvml", self.nvml is not None), ("nvidia-smi", self.proc is not None)) if on)}
 
 
@@ -190,11 +218,14 @@ def run_reference(args, cfg):
             rates.append(r); secs.append(s)
     v = statistics.mean(rates)
     sample = f"routing+grouping on all {cfg.T} tokens, FFN on {nt} seeded tokens per step"
+    # ms_per_step is what one step of this arm took on the clock (a step evaluates the bounded sample); the time
+    # a whole batch would take at the measured rate is an extrapolation and is kept apart
     out = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-           "warmup": args.warmup, "ms_per_step": 1e3 * cfg.T / v, "higher_is_better": True, "scaling": "weak",
+           "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(secs), "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "F": cfg.F, "n": cfg.n, "K": cfg.K,
-                      "F_sh": cfg.F_sh, "sample": sample},
+           "ffn_tokens_per_step": int(nt), "whole_batch_ms_extrapolated": 1e3 * cfg.T / v,
+           "config": {"workload": cfg.name, "variant": "default", "T": cfg.T, "H": cfg.H, "F": cfg.F, "n": cfg.n,
+                      "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam, "sample": sample},
            "cpu_baseline": {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -319,6 +350,238 @@ def run_stack(args, cfg, L, layer0, d_h, dev, rank, world, stream):
             "ms_per_block": ms / args.layers}), flush=True)
 
 
+def build_layer(args, cfg, L, dev, out_dtype=None, like=None):
+    """A PathMoELayer on `dev` for workload L; `like` shares an existing layer's device weights."""
+    from paper_2609_01024_b200 import binding as B
+    mask = np.eye(cfg.n, dtype=np.uint8) if args.variant == "vanilla" else L.mask
+    dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
+    if like is None:
+        wts = tuple(B.to_device(x, dev) for x in (L.w_gate, L.w_up, L.w_down))
+        shared = tuple(B.to_device(x, dev) for x in (L.wsh_gate, L.wsh_up, L.wsh_down)) if cfg.F_sh else None
+    else:
+        wts, shared = (like.w_gate, like.w_up, like.w_down), (like.shared if cfg.F_sh else None)
+    return B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=cfg.F, mask=mask, bias=L.bias,
+                          w_gate=wts[0], w_up=wts[1], w_down=wts[2], shared=shared, max_tokens=cfg.T, in_dtype=dt,
+                          out_dtype=B.PCOMOE_FP32 if out_dtype is None else out_dtype, lam=cfg.lam,
+                          ffn_impl=args.ffn_impl, target_reuse=args.target_reuse, device=dev)
+
+
+def time_stages(layer, cfg, d_logits, d_h, stream, with_router, n_rep, skip):
+    """One continuous run of `n_rep` steps taken stage by stage through the separate entry points, an event at every
+    boundary (no idle gaps between the stages).  Returns the mean and the best time of every stage over the steps
+    after the first `skip`, and the mean time of a whole step."""
+    import torch
+    stage_list = [("router", lambda: layer.router_logits(d_h)), ("route", lambda: layer.route(d_logits)),
+                  ("groups", lambda: layer.build_groups(cfg.T)),
+                  ("stage1_routed", lambda: layer.ffn_stages(d_h, 1)), ("stage1_shared", lambda: layer.ffn_stages(d_h, 2)),
+                  ("stage2_routed", lambda: layer.ffn_stages(d_h, 4)), ("stage2_shared", lambda: layer.ffn_stages(d_h, 8))]
+    stage_list = [(nm, fn) for nm, fn in stage_list
+                  if not ("shared" in nm and not cfg.F_sh) and not (nm == "router" and not with_router)]
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stage_list) + 1)] for _ in range(n_rep)]
+    for i in range(n_rep):
+        marks[i][0].record(stream)
+        for j, (_, fn) in enumerate(stage_list):
+            fn()
+            marks[i][j + 1].record(stream)
+    torch.cuda.synchronize()
+    mean = {nm: statistics.mean(marks[i][j].elapsed_time(marks[i][j + 1]) for i in range(skip, n_rep))
+            for j, (nm, _) in enumerate(stage_list)}
+    best = {nm: min(marks[i][j].elapsed_time(marks[i][j + 1]) for i in range(skip, n_rep))
+            for j, (nm, _) in enumerate(stage_list)}
+    step_ms = statistics.mean(marks[i][0].elapsed_time(marks[i][-1]) for i in range(skip, n_rep))
+    return mean, best, step_ms
+
+
+def dominant_roofline(cfg, work, n_src, stage_ms, peak_tflops, peak_gbs, regime, region, traffic, source):
+    """`roofline` of the dominant kernel (the stage-1 grouped GEMM over the routed groups) in one clock regime:
+    the time and the peak both belong to `regime`."""
+    tc_path = cfg.dtype == "bf16"
+    t = stage_ms["stage1_routed"] * 1e-3
+    if tc_path and cfg.T >= 1024:
+        ach = work["flops_s1"] / t / 1e12
+        return {"bound": "tensor", "achieved": ach, "peak": peak_tflops, "unit": "TFLOP/s", "frac": ach / peak_tflops,
+                "traffic": traffic, "regime": regime, "timed_region": region,
+                "kernel": "stage-1 grouped GEMM over the routed groups (row gather + grouped_gemm_pair_kernel<1>)",
+                "algorithmic": "4*R1*H*F FLOP per launch", "peak_source": source}
+    s1_bytes = (2 if tc_path else 4) * (2 * n_src * cfg.H * cfg.F)
+    ach = s1_bytes / t / 1e9
+    return {"bound": "hbm", "achieved": ach, "peak": peak_gbs, "unit": "GB/s", "frac": ach / peak_gbs,
+            "traffic": traffic, "regime": regime, "timed_region": region,
+            "kernel": "stage-1 grouped GEMM, routed groups (weight streaming, grouped_gemm_kernel<1>)",
+            "algorithmic": "2*n_src*H*F*sizeof(weight) bytes per launch", "peak_source": source}
+
+
+def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, headline):
+    """Everything bench.py reports for one benchmark layer.  `headline`: the configuration the JSON line is about
+    (all extras); otherwise a shorter pass for the `per_config` list."""
+    import torch
+    from paper_2609_01024_b200 import binding as B
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    L = wl.make_layer(cfg)                              # same mask, bias and weights on every rank
+    L.h, L.logits = replicas.rank_inputs(cfg, rank)     # its own batch of tokens
+    layer = build_layer(args, cfg, L, dev)
+    d_logits = torch.from_numpy(L.logits).to(dev)
+    d_h = B.to_device(L.h, dev)
+    if headline and args.layers > 0:
+        run_stack(args, cfg, L, layer, d_h, dev, rank, world, stream)
+        return None
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps ----
+    step = lambda: layer.forward(d_logits, d_h)
+    with_router = headline and args.router >= 0
+    if with_router:
+        w_r, l_a, l_b = wl.make_router_weights(cfg, lora_rank=args.router)
+        layer.set_router(B.to_device(w_r, dev), B.to_device(l_a, dev),
+                         None if l_b is None else torch.from_numpy(l_b).to(dev), 1.0)
+        step = lambda: layer.forward_hidden(d_h)
+        assert not args.graph, "--graph records the logits-in path"
+    if headline and args.graph:
+        step()
+        torch.cuda.synchronize()
+        graph = layer.capture(d_logits, d_h)
+        step = graph.replay
+    for _ in range(args.warmup):
+        step()
+    assert layer.device_status() == 0, "device reported an error during warm-up"
+    if headline and args.profile:
+        for _ in range(args.steps):
+            step()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_run": cfg.name, "steps": args.steps, "status": layer.device_status()}))
+        return None
+    try:
+        uuid = torch.cuda.get_device_properties(dev).uuid
+    except Exception:
+        uuid = None
+    sampler = ClockSampler(local, uuid)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    n0 = B.pcomoe_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = B.pcomoe_launch_count() - n0
+    if headline and args.graph:   # replays do not pass through the library's launch counter: count the captured launches
+        m0 = B.pcomoe_launch_count(); layer.forward(d_logits, d_h); launches = (B.pcomoe_launch_count() - m0) * args.steps
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.window(t_wall0, t_wall1) if rank == 0 else None
+    assert layer.device_status() == 0, "device reported an error during the timed steps"
+    ms_per_step = replicas.max_over_ranks(ms, dev) / args.steps
+    value = replicas.whole_job_tokens_per_s(cfg.T, world, ms_per_step)
+
+    # ---- end to end through the library's host-buffer call (pcomoe_host_pipe_submit): every step copies its logits
+    #      and hidden states from pinned host memory and its y back; the library overlaps the copies of neighbouring
+    #      steps with the kernels.  Once with the fp32 y the parity bar is stated on, once with a bf16 y. ----
+    pin_logits = torch.from_numpy(L.logits).pin_memory()
+    pin_h = (torch.from_numpy(L.h.view(np.int16)).view(torch.bfloat16) if L.h.dtype == np.uint16
+             else torch.from_numpy(L.h)).pin_memory()
+
+    def e2e_of(lay, y_bytes):
+        lay.stream_from_host(pin_logits, pin_h, 3)
+        barrier()
+        t0 = time.perf_counter()
+        y_host = lay.stream_from_host(pin_logits, pin_h, args.steps)
+        torch.cuda.synchronize()
+        v = world * cfg.T * args.steps / replicas.max_over_ranks(time.perf_counter() - t0, dev)
+        assert bool(torch.isfinite(y_host.float()).all())
+        return {"value": v, "unit": UNIT, "h2d_bytes_per_step": int(L.logits.nbytes + L.h.nbytes),
+                "d2h_bytes_per_step": int(cfg.T * cfg.H * y_bytes)}
+    e2e = e2e_of(layer, 4)
+    e2e["y_dtype"] = "f32"
+    e2e["api"] = "pcomoe_host_pipe_submit / pcomoe_host_pipe_wait (C ABI, host pointers), 2 slots"
+    layer._pipe.close(); layer._pipe = None
+    lay16 = build_layer(args, cfg, L, dev, out_dtype=B.PCOMOE_BF16, like=layer)
+    e2e_bf16 = e2e_of(lay16, 2)
+    e2e_bf16["y_dtype"] = "bf16"
+    lay16.close()
+    del lay16
+
+    # ---- per-kernel timing for the roofline: dominant kernel = stage-1 grouped GEMM ----
+    stats = layer.groups.stats.cpu().numpy()
+    R1 = int(stats[0])
+    n_src = cfg.n - int(stats[4]); n_tgt = cfg.n - int(stats[5])
+    work = algorithmic_work(cfg, R1, n_src, n_tgt)
+    pk = peaks()
+    traffic = ncu_traffic_stage1(config_index) if not args.shape and args.variant == "default" else None
+    # (a) burst regime: the GPU idles for a second, then a short run of steps; divided by the burst peak
+    torch.cuda.synchronize()
+    time.sleep(1.0)
+    n_rep = 3 + args.steps
+    burst_mean, burst_best, burst_step = time_stages(layer, cfg, d_logits, d_h, stream, with_router, n_rep, 3)
+    region = f"{n_rep} steps taken stage by stage after 1 s of idle, about {burst_step * n_rep:.0f} ms; mean over the last {n_rep - 3}"
+    roofline = dominant_roofline(cfg, work, n_src, burst_mean, pk["bf16_tflops"], pk["hbm_gbs"], "burst", region, traffic,
+                                 pk["source"] + " burst bf16 GEMM / copy bandwidth")
+    roofline["frac_best_step"] = roofline["frac"] * burst_mean["stage1_routed"] / burst_best["stage1_routed"]
+    # (b) sustained regime: >= 2 s of back-to-back steps first, then the stage-by-stage run continues without a gap;
+    #     divided by the sustained peak
+    t_s0 = time.time()
+    n_pre = max(10, int(2000.0 / ms_per_step))
+    es0, es1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(n_pre // 2):
+        step()
+    es0.record(stream)
+    for _ in range(n_pre - n_pre // 2):
+        step()
+    es1.record(stream)
+    n_sus = max(10, int(500.0 / ms_per_step))
+    sus_mean, _, sus_step = time_stages(layer, cfg, d_logits, d_h, stream, with_router, n_sus, 0)
+    t_s1 = time.time()
+    ms_sustained = es0.elapsed_time(es1) / (n_pre - n_pre // 2)
+    region = (f"{n_pre} back-to-back steps ({n_pre * ms_sustained / 1e3:.1f} s), then {n_sus} steps taken stage by stage "
+              f"without a gap; mean over those")
+    roofline_sus = dominant_roofline(cfg, work, n_src, sus_mean, pk["bf16_tflops_sustained"], pk["hbm_gbs"], "sustained",
+                                     region, traffic, pk["source"] + " sustained bf16 GEMM / copy bandwidth")
+    roofline_sus["ms_per_step"] = ms_sustained
+    roofline_sus["stage_ms"] = sus_mean
+    if rank == 0:
+        roofline_sus["clocks"] = sampler.window(t_s0, t_s1)
+        sampler.stop()
+    assert layer.device_status() == 0
+    # whole-layer roofline time: max(FLOPs / tensor peak, bytes / HBM peak), like for like in each regime
+    t_roof = lambda tf, gbs: max(work["flops"] / (tf * 1e12), work["bytes"] / (gbs * 1e9))
+    layer_roofline = {"flops": work["flops"], "bytes": work["bytes"],
+                      "frac_burst": t_roof(pk["bf16_tflops"], pk["hbm_gbs"]) / (ms_per_step * 1e-3),
+                      "frac_sustained": t_roof(pk["bf16_tflops_sustained"], pk["hbm_gbs"]) / (ms_sustained * 1e-3),
+                      "frac_of_nominal_2.25PF_8TBs": t_roof(2250.0, 8000.0) / (ms_per_step * 1e-3),
+                      "note": "frac_burst: the headline loop's ms_per_step (tens of ms from warm clocks) over the burst "
+                              "peaks; frac_sustained: ms_per_step after 1 s of continuous steps over the sustained peak"}
+    tc_path = cfg.dtype == "bf16"
+    res = {"ms_per_step": ms_per_step, "value": value, "e2e": e2e, "e2e_bf16_y": e2e_bf16, "launches": int(launches),
+           "clocks": clocks, "roofline": roofline, "roofline_sustained": roofline_sus, "layer_roofline": layer_roofline,
+           "stage_ms": burst_mean, "dtype": "bf16" if tc_path else "f32",
+           "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
+                      "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam,
+                      "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(headline and args.graph),
+                      "target_reuse": int(args.target_reuse),
+                      "stage2_rows_over_P": int(stats[1]) / (cfg.T * cfg.K),
+                      "router_in_step": (f"yes (rank-{args.router} gate adaptation)" if with_router and args.router > 0 else
+                                         "yes" if with_router else "no (logits are an input)"),
+                      "parallelism": f"token-dp{world} (replicas, no collective)",
+                      "l2": "inputs larger than L2 (weights are streamed every step)" if work["weight_bytes"] > 126e6
+                            else "working set fits L2; not a performance target"}}
+    if headline and args.sweep_density and world == 1 and rank == 0:
+        res["density_sweep"] = density_sweep(args, cfg, L, layer, d_logits, d_h, dev, stream)
+    if headline and not args.no_cpu_baseline and world == 1 and rank == 0:
+        n_cpu = args.cpu_tokens
+        if n_cpu <= 0:   # probe with a few tokens per thread, then size the sample for about 20 s
+            r0, _, s0, nt0 = oracle_sample_rate(cfg, L, 32)
+            n_cpu = int(max(32, min(cfg.T, 20.0 * r0)))
+        r, thr, secs, nt = oracle_sample_rate(cfg, L, n_cpu)
+        res["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": thr, "kind": "oracle",
+                               "sample": f"routing+grouping on all {cfg.T} tokens, FFN on {nt} seeded tokens ({secs:.1f} s)"}
+    layer.close()
+    del layer, d_logits, d_h, L
+    torch.cuda.empty_cache()
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -334,6 +597,8 @@ def main():
                     help="only run warm-up + steps of the device-resident hot path, print a short line and exit")
     ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the per_config list (the other prefill-sized layers and the decode layer, timed after the headline)")
     ap.add_argument("--router", type=int, default=-1,
                     help="r >= 0: the timed step starts from hidden states (router GEMM with a rank-r gate adaptation, "
                          "0 = none, in front of the path gate); default -1: logits are an input, as the metric is quoted")
@@ -364,7 +629,6 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2609_01024_b200 import binding as B
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -375,25 +639,7 @@ def main():
     dev = f"cuda:{local}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
-
-    # Every rank holds a replica of the weights and its own batch of T tokens (token data parallel,
-    # no collective on the data path); rank r draws its tokens with seed + 100*r.
-    L = wl.make_layer(cfg)                              # same mask, bias and weights on every rank
-    L.h, L.logits = replicas.rank_inputs(cfg, rank)     # its own batch of tokens
-    mask = np.eye(cfg.n, dtype=np.uint8) if args.variant == "vanilla" else L.mask
-    dt = B.PCOMOE_FP32 if cfg.dtype == "f32" else B.PCOMOE_BF16
-    layer = B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=cfg.F, mask=mask, bias=L.bias,
-                           w_gate=B.to_device(L.w_gate, dev), w_up=B.to_device(L.w_up, dev),
-                           w_down=B.to_device(L.w_down, dev),
-                           shared=tuple(B.to_device(x, dev) for x in (L.wsh_gate, L.wsh_up, L.wsh_down)) if cfg.F_sh else None,
-                           max_tokens=cfg.T, in_dtype=dt, lam=cfg.lam, ffn_impl=args.ffn_impl,
-                           target_reuse=args.target_reuse, device=dev)
-    d_logits = torch.from_numpy(L.logits).to(dev)
-    d_h = B.to_device(L.h, dev)
     stream = torch.cuda.current_stream()
-    if args.layers > 0:
-        run_stack(args, cfg, L, layer, d_h, dev, rank, world, stream)
-        return
 
     def barrier():
         torch.cuda.synchronize()
@@ -401,149 +647,39 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing: W warm-up steps, then exactly K timed steps ----
-    step = lambda: layer.forward(d_logits, d_h)
-    if args.router >= 0:
-        w_r, l_a, l_b = wl.make_router_weights(cfg, lora_rank=args.router)
-        layer.set_router(B.to_device(w_r, dev), B.to_device(l_a, dev),
-                         None if l_b is None else torch.from_numpy(l_b).to(dev), 1.0)
-        step = lambda: layer.forward_hidden(d_h)
-        assert not args.graph, "--graph records the logits-in path"
-    if args.graph:
-        step()
-        torch.cuda.synchronize()
-        graph = layer.capture(d_logits, d_h)
-        step = graph.replay
-    for _ in range(args.warmup):
-        step()
-    assert layer.device_status() == 0, "device reported an error during warm-up"
-    if args.profile:
-        for _ in range(args.steps):
-            step()
-        torch.cuda.synchronize()
-        print(json.dumps({"profile_run": cfg.name, "steps": args.steps, "status": layer.device_status()}))
-        return
-    try:
-        uuid = torch.cuda.get_device_properties(dev).uuid
-    except Exception:
-        uuid = None
-    sampler = ClockSampler(local, uuid)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    barrier()
-    n0 = B.pcomoe_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_wall0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    t_wall1 = time.time()
-    launches = B.pcomoe_launch_count() - n0
-    if args.graph:   # replays do not pass through the library's launch counter: count the captured launches
-        m0 = B.pcomoe_launch_count(); layer.forward(d_logits, d_h); launches = (B.pcomoe_launch_count() - m0) * args.steps
-    ms = e0.elapsed_time(e1)
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    assert layer.device_status() == 0, "device reported an error during the timed steps"
-    ms_per_step = replicas.max_over_ranks(ms, dev) / args.steps
-    value = replicas.whole_job_tokens_per_s(cfg.T, world, ms_per_step)
-
-    # ---- end to end from pinned host buffers: every step copies its inputs host->device and its y device->host;
-    #      the copies run on their own streams, overlapped with the kernels of the neighbouring steps ----
-    pin_logits = torch.from_numpy(L.logits).pin_memory()
-    pin_h = (torch.from_numpy(L.h.view(np.int16)).view(torch.bfloat16) if L.h.dtype == np.uint16
-             else torch.from_numpy(L.h)).pin_memory()
-    layer.stream_from_host(pin_logits, pin_h, 3)
-    barrier()
-    t0 = time.perf_counter()
-    y_host = layer.stream_from_host(pin_logits, pin_h, args.steps)
-    torch.cuda.synchronize()
-    e2e_value = world * cfg.T * args.steps / replicas.max_over_ranks(time.perf_counter() - t0, dev)
-    h2d = L.logits.nbytes + L.h.nbytes
-    d2h = cfg.T * cfg.H * 4
-    assert layer.device_status() == 0 and bool(torch.isfinite(y_host).all())
-
-    # ---- per-kernel timing for the roofline: dominant kernel = stage-1 grouped GEMM ----
-    stats = layer.groups.stats.cpu().numpy()
-    R1 = int(stats[0])
-    n_src = cfg.n - int(stats[4]); n_tgt = cfg.n - int(stats[5])
-    work = algorithmic_work(cfg, R1, n_src, n_tgt)
-    # Stage times are taken inside a continuous run of steps (no idle gaps between the stages: the clocks and the
-    # cache state are those of the timed loop); every step goes stage by stage through the separate entry points
-    # with an event at each boundary.
-    stage_list = [("router", lambda: layer.router_logits(d_h)), ("route", lambda: layer.route(d_logits)),
-                  ("groups", lambda: layer.build_groups(cfg.T)),
-                  ("stage1_routed", lambda: layer.ffn_stages(d_h, 1)), ("stage1_shared", lambda: layer.ffn_stages(d_h, 2)),
-                  ("stage2_routed", lambda: layer.ffn_stages(d_h, 4)), ("stage2_shared", lambda: layer.ffn_stages(d_h, 8))]
-    stage_list = [(nm, fn) for nm, fn in stage_list
-                  if not ("shared" in nm and not cfg.F_sh) and not (nm == "router" and args.router < 0)]
-    n_rep = 3 + args.steps
-    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stage_list) + 1)] for _ in range(n_rep)]
-    torch.cuda.synchronize()
-    time.sleep(1.0)        # start from the idle power state the headline loop started from
-    for i in range(n_rep):
-        marks[i][0].record(stream)
-        for j, (_, fn) in enumerate(stage_list):
-            fn()
-            marks[i][j + 1].record(stream)
-    torch.cuda.synchronize()
-    stage_ms = {nm: statistics.mean(marks[i][j].elapsed_time(marks[i][j + 1]) for i in range(3, n_rep))
-                for j, (nm, _) in enumerate(stage_list)}
-    pk = peaks()
-    tc_path = cfg.dtype == "bf16"
-    if tc_path and cfg.T >= 1024:
-        # prefill-sized: tensor-bound; stage-1 routed GEMM is the dominant kernel
-        ach = work["flops_s1"] / (stage_ms["stage1_routed"] * 1e-3) / 1e12
-        peak = pk["bf16_tflops_sustained"]
-        roofline = {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                    "traffic": NCU_TRAFFIC_STAGE1.get(args.config) if not args.shape and args.variant == "default" else None,
-                    "kernel": "stage-1 grouped GEMM over the routed groups (row gather + grouped_gemm_pair_kernel<1>)",
-                    "peak_source": pk["source"] + " sustained bf16 (kernel timed inside a loop of steps)"}
-    else:
-        # decode-sized / tiny: weight streaming; report the two GEMM stages' bytes against HBM
-        s1_bytes = 2 * (2 * n_src * cfg.H * cfg.F) if tc_path else 4 * (2 * n_src * cfg.H * cfg.F)
-        ach = s1_bytes / (stage_ms["stage1_routed"] * 1e-3) / 1e9
-        peak = pk["hbm_gbs"]
-        roofline = {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                    "traffic": NCU_TRAFFIC_STAGE1.get(args.config) if not args.shape and args.variant == "default" else None,
-                    "kernel": "stage-1 grouped GEMM, routed groups (weight streaming, grouped_gemm_kernel<1>)",
-                    "peak_source": pk["source"] + " copy bandwidth"}
-    # whole-layer roofline time: max(FLOPs / tensor peak, bytes / HBM peak)
-    t_roof_meas = max(work["flops"] / (pk["bf16_tflops_sustained"] * 1e12), work["bytes"] / (pk["hbm_gbs"] * 1e9))
-    t_roof_nominal = max(work["flops"] / 2.25e15, work["bytes"] / 8e12)
-
-    out = None
-    if rank == 0:
-        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-               "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-               "vs_baseline": None, "dtype": "bf16" if tc_path else "f32", "data": "synthetic",
-               "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
-                          "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh, "mask_p": cfg.mask_p, "lambda": cfg.lam,
-                          "R1_over_P": R1 / (cfg.T * cfg.K), "cuda_graph": bool(args.graph), "target_reuse": int(args.target_reuse),
-                          "stage2_rows_over_P": int(stats[1]) / (cfg.T * cfg.K),
-                          "router_in_step": (f"yes (rank-{args.router} gate adaptation)" if args.router > 0 else
-                                             "yes" if args.router == 0 else "no (logits are an input)"),
-                          "parallelism": f"token-dp{world} (replicas, no collective)",
-                          "l2": "inputs larger than L2 (weights are streamed every step)" if work["weight_bytes"] > 126e6
-                                else "working set fits L2; not a performance target"},
-               "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
-               "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
-               "layer_roofline": {"flops": work["flops"], "bytes": work["bytes"],
-                                  "frac_of_measured": t_roof_meas / (ms_per_step * 1e-3),
-                                  "frac_of_nominal_2.25PF_8TBs": t_roof_nominal / (ms_per_step * 1e-3)},
-               "stage_ms": stage_ms}
-        if args.sweep_density and world == 1:
-            out["density_sweep"] = density_sweep(args, cfg, L, layer, d_logits, d_h, dev, stream)
-        if not args.no_cpu_baseline and world == 1:
-            n_cpu = args.cpu_tokens
-            if n_cpu <= 0:   # probe with a few tokens per thread, then size the sample for about 20 s
-                r0, _, s0, nt0 = oracle_sample_rate(cfg, L, 32)
-                n_cpu = int(max(32, min(cfg.T, 20.0 * r0)))
-            r, thr, secs, nt = oracle_sample_rate(cfg, L, n_cpu)
-            out["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": thr, "kind": "oracle",
-                                   "sample": f"routing+grouping on all {cfg.T} tokens, FFN on {nt} seeded tokens ({secs:.1f} s)"}
+    # Every rank holds a replica of the weights and its own batch of T tokens (token data parallel,
+    # no collective on the data path); rank r draws its tokens with seed + 100*r.
+    res = measure_config(args, cfg, args.config, dev, rank, world, stream, barrier, headline=True)
+    if res is not None and rank == 0:
+        out = {"metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": res["dtype"], "data": "synthetic", "config": res["config"],
+               "e2e": res["e2e"], "e2e_bf16_y": res["e2e_bf16_y"], "gpu_launches": res["launches"],
+               "clocks": res["clocks"], "roofline": res["roofline"], "roofline_sustained": res["roofline_sustained"],
+               "layer_roofline": res["layer_roofline"], "stage_ms": res["stage_ms"]}
+        for k in ("density_sweep", "cpu_baseline"):
+            if k in res:
+                out[k] = res[k]
+    # The other benchmark layers, timed the same way after the headline (one GPU only: the scaling runs repeat the
+    # headline configuration at every N).
+    plain = (args.config == 2 and not args.shape and args.variant == "default" and args.router < 0 and not args.graph
+             and args.layers == 0 and not args.profile and args.target_reuse == 0 and args.ffn_impl == 0)
+    if res is not None and world == 1 and plain and not args.no_per_config:
+        per = {}
+        for ci in (3, 4, 5):
+            r = measure_config(args, wl.CONFIGS[ci], ci, dev, rank, world, stream, barrier, headline=False)
+            per[str(ci)] = {"workload": r["config"]["workload"], "T": wl.CONFIGS[ci].T, "ms_per_step": r["ms_per_step"],
+                            "tokens_per_s": r["value"], "R1_over_P": r["config"]["R1_over_P"],
+                            "e2e_tokens_per_s": r["e2e"]["value"], "e2e_bf16_y_tokens_per_s": r["e2e_bf16_y"]["value"],
+                            "gpu_launches": r["launches"], "stage_ms": r["stage_ms"],
+                            "roofline": {k: r["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "traffic")},
+                            "roofline_sustained": {k: r["roofline_sustained"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "ms_per_step")},
+                            "layer_frac_burst": r["layer_roofline"]["frac_burst"],
+                            "layer_frac_sustained": r["layer_roofline"]["frac_sustained"],
+                            "layer_frac_of_nominal_2.25PF_8TBs": r["layer_roofline"]["frac_of_nominal_2.25PF_8TBs"],
+                            "clocks": r["clocks"]}
+        out["per_config"] = per
+    if res is not None and rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.barrier()

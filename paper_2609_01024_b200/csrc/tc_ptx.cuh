@@ -44,7 +44,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 }
 // Bounded wait: gives up after `limit_ns` (the library-wide limit, see wait_limit_ns(); the kernels carry it in
 // their parameters).  Returns false when the CTA is giving up (this or another role timed out).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t it = 1; it < (1u << 24); ++it) {
@@ -54,6 +54,21 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
   }
   *abort_flag = 1;
   return false;
+}
+
+// The common case - the phase has already completed - is one non-blocking probe in line; only a wait that
+// really has to wait pays for the call.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  if (ok) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, limit_ns);
 }
 
 // What a CTA does once one of its waits has run out: record the timeout in the status word, then give the

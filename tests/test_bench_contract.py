@@ -16,6 +16,8 @@ def test_reference_arm_prints_the_contract_line():
     assert line["impl"] == "reference" and line["metric"] == "path_moe_layer_tokens_per_s" and line["unit"] == "tokens/s"
     assert line["higher_is_better"] is True and line["steps"] == 2 and line["warmup"] == 1 and line["n_gpus"] == 1
     assert line["value"] > 0 and line["ms_per_step"] > 0
+    # ms_per_step is the measured time of a step (a bounded sample), the whole-batch figure is kept apart
+    assert line["ffn_tokens_per_step"] > 0 and line["whole_batch_ms_extrapolated"] > 0
     assert line["config"]["workload"].startswith("cfg1")
     cb = line["cpu_baseline"]
     assert cb["kind"] == "oracle" and cb["cores"] >= 1 and cb["value"] == line["value"] and cb["sample"]

@@ -51,8 +51,9 @@ def test_benchmark_layer_matches_oracle(G, oracle, full_reference, idx):
 
 @pytest.mark.parametrize("idx", [5, 3, 4, 2])
 def test_benchmark_layer_bf16_output_matches_oracle(G, full_reference, idx):
-    """out_dtype = bf16: the fp32 sum rounded once at the end.  Same bars as the fp32 output: the extra half ulp
-    of bf16 (at most 2^-7 for |y| < 4) stays inside the max-abs bound, and adds about 1.1e-3 to the relative L2."""
+    """out_dtype = bf16: the fp32 sum rounded once at the end.  The relative-L2 bar is the fp32 output's (the
+    rounding adds about 1.1e-3); element by element the bar is the fp32 output's 2e-2 plus the half ulp of the
+    final rounding, 2^-8 |y|."""
     import torch
     cfg, L, rs, rt, rw, yr = full_reference(idx)
     layer = G.make_gpu_layer(cfg, L, out_dtype=G.B.PCOMOE_BF16)
@@ -60,5 +61,5 @@ def test_benchmark_layer_bf16_output_matches_oracle(G, full_reference, idx):
     assert layer.device_status() == 0 and y.dtype == torch.bfloat16
     y = y.float().cpu().numpy()
     assert np.array_equal(layer.path_src[:cfg.T].cpu().numpy(), rs)
-    assert np.abs(yr).max() < 4.0            # the premise of the half-ulp bound above
-    G.check_output(y, yr, max_abs=2e-2, rel_l2=5e-3)
+    assert np.all(np.abs(y - yr) <= 2e-2 + np.abs(yr) / 256.0)
+    G.check_output(y, yr, max_abs=2e-2 + np.abs(yr).max() / 256.0, rel_l2=5e-3)
