@@ -92,29 +92,30 @@ struct TileInfo {
 // that CTAs working at the same time share one slice of the group's weights.
 struct TileWalker {
   const int32_t *tb, *ro;      // [2][kMaxExperts + 2] each
-  int nt[2], G[2], mo[2], nseg;
-  int seg, g, seg_first;       // current segment, group, and the first tile id of the segment
-  __device__ int seg_tiles(int s) const { return tb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
-  __device__ int total() const {
-    int t = 0;
-    for (int s = 0; s < nseg; ++s) t += seg_tiles(s);
-    return t;
+  int nt0, nt1, G0, G1, mo0, mo1, nseg;   // per segment (scalars: indexed arrays would live in local memory)
+  int seg, g;                  // current segment and group
+  int tiles0;                  // tiles of segment 0
+  __device__ void init() {
+    seg = 0; g = 0;
+    tiles0 = tb[G0] * nt0;
   }
+  __device__ int total() const { return tiles0 + (nseg > 1 ? tb[(kMaxExperts + 2) + G1] * nt1 : 0); }
+  __device__ int seg_of(int tile) const { return (nseg > 1 && tile >= tiles0) ? 1 : 0; }
   __device__ TileInfo at(int tile) {
-    while (seg + 1 < nseg && tile >= seg_first + seg_tiles(seg)) {
-      seg_first += seg_tiles(seg);
-      ++seg;
+    if (seg == 0 && nseg > 1 && tile >= tiles0) {
+      seg = 1;
       g = 0;
     }
     const int32_t *b = tb + seg * (kMaxExperts + 2), *r = ro + seg * (kMaxExperts + 2);
-    const int n_t = nt[seg], local_seg = tile - seg_first;
-    while (g + 1 < G[seg] && local_seg >= b[g + 1] * n_t) ++g;
+    const int n_t = seg ? nt1 : nt0, Gs = seg ? G1 : G0, m_out = seg ? mo1 : mo0;
+    const int local_seg = tile - (seg ? tiles0 : 0);
+    while (g + 1 < Gs && local_seg >= b[g + 1] * n_t) ++g;
     TileInfo t;
     const int mt = b[g + 1] - b[g];
     const int local = local_seg - b[g] * n_t;
     t.seg = seg;
     t.g = g;
-    if (mo[seg]) {
+    if (m_out) {
       t.m_idx = local / n_t;
       t.n_idx = local - t.m_idx * n_t;
     } else {
@@ -410,13 +411,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
 
   TileWalker walk;
   walk.tb = s_tb; walk.ro = s_ro; walk.nseg = p.nseg;
-  for (int sg = 0; sg < 2; ++sg) {
-    walk.nt[sg] = p.seg[sg].nt;
-    walk.mo[sg] = p.seg[sg].m_outer;
-    walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
-  }
-  walk.seg = 0; walk.g = 0; walk.seg_first = 0;
+  walk.nt0 = p.seg[0].nt; walk.nt1 = p.seg[1].nt;
+  walk.mo0 = p.seg[0].m_outer; walk.mo1 = p.seg[1].m_outer;
+  walk.G0 = p.seg[0].tile_base ? p.seg[0].G : 1; walk.G1 = p.seg[1].tile_base ? p.seg[1].G : 1;
+  walk.init();
   const int total = walk.total();
+  const int kb0 = p.seg[0].kb, kb1 = p.seg[1].kb;
 
   if (warp == 0) {
     // ---------------- producer: TMA into the ring ----------------
@@ -454,8 +454,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_const
       uint32_t phase = 0, acc_phase = 0;
       bool alive = true;
       for (int tile = blockIdx.x; tile < total && alive; tile += gridDim.x) {
-        const TileInfo t = walk.at(tile);
-        const int nkb = p.seg[t.seg].kb;
+        const int nkb = walk.seg_of(tile) ? kb1 : kb0;   // all the issuer needs to know about the tile
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_ns)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
@@ -581,30 +580,31 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 // run fastest.  CTA `rank` of the pair owns m-tile 2*pair + rank of the group.
 struct PairWalker {
   const int32_t *tb, *ro, *pb;   // [2][kMaxExperts + 2] each: m-tile prefix, row offsets, pair prefix
-  int nt[2], G[2], mo[2], nseg;
-  int seg, g, seg_first;
-  __device__ int seg_tiles(int s) const { return pb[s * (kMaxExperts + 2) + G[s]] * nt[s]; }
-  __device__ int total() const {
-    int t = 0;
-    for (int s = 0; s < nseg; ++s) t += seg_tiles(s);
-    return t;
+  int nt0, nt1, G0, G1, mo0, mo1, nseg;   // per segment (scalars: indexed arrays would live in local memory)
+  int seg, g;
+  int tiles0;                    // pair tiles of segment 0
+  __device__ void init() {
+    seg = 0; g = 0;
+    tiles0 = pb[G0] * nt0;
   }
+  __device__ int total() const { return tiles0 + (nseg > 1 ? pb[(kMaxExperts + 2) + G1] * nt1 : 0); }
+  __device__ int seg_of(int tile) const { return (nseg > 1 && tile >= tiles0) ? 1 : 0; }
   __device__ TileInfo at(int tile, int rank) {
-    while (seg + 1 < nseg && tile >= seg_first + seg_tiles(seg)) {
-      seg_first += seg_tiles(seg);
-      ++seg;
+    if (seg == 0 && nseg > 1 && tile >= tiles0) {
+      seg = 1;
       g = 0;
     }
     const int o = seg * (kMaxExperts + 2);
     const int32_t *b = tb + o, *r = ro + o, *q = pb + o;
-    const int n_t = nt[seg], local_seg = tile - seg_first;
-    while (g + 1 < G[seg] && local_seg >= q[g + 1] * n_t) ++g;
+    const int n_t = seg ? nt1 : nt0, Gs = seg ? G1 : G0, m_out = seg ? mo1 : mo0;
+    const int local_seg = tile - (seg ? tiles0 : 0);
+    while (g + 1 < Gs && local_seg >= q[g + 1] * n_t) ++g;
     TileInfo t;
     const int np = q[g + 1] - q[g];
     const int local = local_seg - q[g] * n_t;
     t.seg = seg;
     t.g = g;
-    if (mo[seg]) {
+    if (m_out) {
       const int pr = local / n_t;
       t.n_idx = local - pr * n_t;
       t.m_idx = 2 * pr + rank;
@@ -619,7 +619,9 @@ struct PairWalker {
   }
 };
 
-template <int STAGE, bool MERGE = false, int NST = STAGES2>
+// A ring stage holds KSUB k-blocks (KSUB x 32 KB per CTA): with KSUB = 2 the barrier round trips, the producer's
+// wake-ups and the issuer's waits happen once per 128 columns of K instead of once per 64.
+template <int STAGE, bool MERGE = false, int NST = STAGES2, int KSUB = 1>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                          const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmA1,
@@ -696,13 +698,12 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
 
   PairWalker walk;
   walk.tb = s_tb; walk.ro = s_ro; walk.pb = s_pb; walk.nseg = p.nseg;
-  for (int sg = 0; sg < 2; ++sg) {
-    walk.nt[sg] = p.seg[sg].nt;
-    walk.mo[sg] = p.seg[sg].m_outer;
-    walk.G[sg] = p.seg[sg].tile_base ? p.seg[sg].G : 1;
-  }
-  walk.seg = 0; walk.g = 0; walk.seg_first = 0;
+  walk.nt0 = p.seg[0].nt; walk.nt1 = p.seg[1].nt;
+  walk.mo0 = p.seg[0].m_outer; walk.mo1 = p.seg[1].m_outer;
+  walk.G0 = p.seg[0].tile_base ? p.seg[0].G : 1; walk.G1 = p.seg[1].tile_base ? p.seg[1].G : 1;
+  walk.init();
   const int total = walk.total();
+  const int kb0 = p.seg[0].kb, kb1 = p.seg[1].kb;
 
   if (warp == 0) {
     // ---------------- producer (both CTAs): own A rows and own half of B ----------------
@@ -725,13 +726,16 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
           mB = t.seg ? &tmB1 : &tmB0;
           b_row = t.g * S.b_group_rows + t.n_idx * 256 + (int)rank * 128;
         }
-        for (int kb = 0; kb < S.kb; ++kb) {
+        for (int kb = 0; kb < S.kb; kb += KSUB) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_ns)) { alive = false; break; }
-          const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
+          const uint32_t s0 = ring + stage * (KSUB * STAGE2_BYTES);
           const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
-          tma_load_2d_pair(sa, mA, kb * BK, a_row, lead_full);
-          tma_load_2d_pair(sb, mB, kb * BK, b_row, lead_full);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * KSUB * STAGE2_BYTES);
+#pragma unroll
+          for (int j = 0; j < KSUB; ++j) {
+            tma_load_2d_pair(s0 + j * STAGE2_BYTES, mA, (kb + j) * BK, a_row, lead_full);
+            tma_load_2d_pair(s0 + j * STAGE2_BYTES + HALF_BYTES, mB, (kb + j) * BK, b_row, lead_full);
+          }
           if (++stage == NST) { stage = 0; phase ^= 1u; }
         }
       }
@@ -744,19 +748,21 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_
       uint32_t phase = 0, acc_phase = 0;
       bool alive = true;
       for (int tile = pair_id; tile < total && alive; tile += n_pairs) {
-        const TileInfo t = walk.at(tile, 0);
-        const int nkb = p.seg[t.seg].kb;
+        const int nkb = walk.seg_of(tile) ? kb1 : kb0;   // all the issuer needs to know about the tile
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_ns)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = 0; kb < nkb; kb += KSUB) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.wait_ns)) { alive = false; break; }
           tc_fence_after();
-          const uint32_t sa = ring + stage * STAGE2_BYTES, sb = sa + HALF_BYTES;
-          const uint64_t da = umma_desc(sa), db = umma_desc(sb);
+          const uint32_t s0 = ring + stage * (KSUB * STAGE2_BYTES);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            umma_bf16_pair(d_tmem, da + 2u * k, db + 2u * k, (kb | k) != 0 ? 1u : 0u);
+          for (int j = 0; j < KSUB; ++j) {
+            const uint64_t da = umma_desc(s0 + j * STAGE2_BYTES), db = umma_desc(s0 + j * STAGE2_BYTES + HALF_BYTES);
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k)
+              umma_bf16_pair(d_tmem, da + 2u * k, db + 2u * k, (kb | j | k) != 0 ? 1u : 0u);
+          }
           umma_commit_pair(empty_bar(stage));
           if (++stage == NST) { stage = 0; phase ^= 1u; }
         }
@@ -863,6 +869,8 @@ static_assert((size_t)STAGES2 * STAGE2_BYTES + 1024 == kSmemDyn, "both kernels u
 // routing, grouping and gather kernels running on another stream at the same time fit on the same SMs (the
 // shared expert needs nothing from them).  Device-side problems go to the router's status word: the grouping
 // step running beside this launch clears the layer's own word.
+constexpr int kPairSub = 2;                        // k-blocks per ring stage of the stage-1 pair kernel (measured: stage 1
+constexpr int kPairStages = STAGES2 / kPairSub;    // 0.5-2 % faster with three stages of 64 KB, stage 2 no faster)
 constexpr int kSideStages = 4;
 constexpr size_t kSmemSide = (size_t)kSideStages * STAGE2_BYTES + 1024;
 
@@ -922,10 +930,10 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
   if (attr_once.first_use(L->device)) {
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
-    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, false, kPairStages, kPairSub>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
-    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
+    PCOMOE_CUDA_TRY(cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, true, kPairStages, kPairSub>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemDyn));
     attr_once.done(L->device);
   }
   const bool pair = use_cta_pairs(L, T);
@@ -984,8 +992,8 @@ pcomoe_status launch_ffn_tc(const pcomoe_layer *L, int32_t T, const void *h, con
       p.zero_ptr = reinterpret_cast<float4 *>(y);
       p.zero_vec4 = (int64_t)T * H / 4;
     }
-    auto k3 = merge ? (pair ? grouped_gemm_pair_kernel<1, true> : grouped_gemm_kernel<1, true>)
-                    : (pair ? grouped_gemm_pair_kernel<1, false> : grouped_gemm_kernel<1, false>);
+    auto k3 = merge ? (pair ? grouped_gemm_pair_kernel<1, true, kPairStages, kPairSub> : grouped_gemm_kernel<1, true>)
+                    : (pair ? grouped_gemm_pair_kernel<1, false, kPairStages, kPairSub> : grouped_gemm_kernel<1, false>);
     PCOMOE_CUDA_TRY(launch_pdl(k3, dim3(grid1), dim3(kThreads), kSmemDyn, st, mA[0], mB[0], mC[0], mA[1], mB[1], mC[1], p));
     count_launch();
   }
