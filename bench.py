@@ -444,8 +444,11 @@ def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, h
         step()
     assert layer.device_status() == 0, "device reported an error during warm-up"
     if headline and args.profile:
-        for _ in range(args.steps):
-            step()
+        if args.profile == "stages":
+            time_stages(layer, cfg, d_logits, d_h, stream, with_router, args.steps, 0)
+        else:
+            for _ in range(args.steps):
+                step()
         torch.cuda.synchronize()
         print(json.dumps({"profile_run": cfg.name, "steps": args.steps, "status": layer.device_status()}))
         return None
@@ -582,6 +585,55 @@ def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, h
     return res
 
 
+def run_tp(args, cfg, dev, rank, world, stream, barrier):
+    """F-sliced tensor parallelism (--tp): every rank holds 1/N of every expert's intermediate width (tile-aligned
+    slices) and runs the whole path on the SAME batch of tokens; routing and grouping are replicated; the one
+    exchange step is a reduce-scatter of the partial outputs over NCCL (each rank ends with the complete y of its
+    T/N tokens).  Strong scaling: the batch is fixed, so value = T tokens / step time."""
+    import torch
+    from paper_2609_01024_b200 import binding as B
+    from paper_2609_01024_b200 import tensor_parallel as tp
+    L = wl.make_layer(cfg)                                  # same tokens, mask, bias on every rank
+    wg, wu, wd = tp.shard_expert_weights(L.w_gate, L.w_up, L.w_down, world, rank)
+    sh = tp.shard_shared_weights(L.wsh_gate, L.wsh_up, L.wsh_down, world, rank) if cfg.F_sh else None
+    Fg = wg.shape[1]
+    layer = B.PathMoELayer(n_experts=cfg.n, top_k=cfg.K, hidden=cfg.H, ffn=Fg, mask=L.mask, bias=L.bias,
+                           w_gate=B.to_device(wg, dev), w_up=B.to_device(wu, dev), w_down=B.to_device(wd, dev),
+                           shared=tuple(B.to_device(x, dev) for x in sh) if sh else None, max_tokens=cfg.T,
+                           lam=cfg.lam, ffn_impl=args.ffn_impl, device=dev)
+    d_logits, d_h = torch.from_numpy(L.logits).to(dev), B.to_device(L.h, dev)
+
+    def step():
+        y = layer.forward(d_logits, d_h)
+        return tp.reduce_scatter_rows(y)[0] if world > 1 else y
+    for _ in range(args.warmup):
+        step()
+    assert layer.device_status() == 0
+    barrier()
+    n0 = B.pcomoe_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    launches = B.pcomoe_launch_count() - n0
+    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+    assert layer.device_status() == 0
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": cfg.T / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16" if cfg.dtype != "f32" else "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "F": cfg.F, "n": cfg.n, "K": cfg.K, "F_sh": cfg.F_sh,
+                       "parallelism": f"tp{world} (F-sliced experts, replicated routing, one reduce-scatter of y)",
+                       "slice_of_rank0": list(tp.slice_bounds(cfg.F, world, 0)),
+                       "l2": "inputs larger than L2 (weights are streamed every step)"},
+            "gpu_launches": int(launches),
+            "exchange": {"collective": "reduce_scatter (NCCL)" if world > 1 else "none",
+                         "bytes_per_rank_per_step": int(cfg.T * cfg.H * 4 * (world - 1) / max(world, 1))}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -593,8 +645,10 @@ def main():
                     help="tokens of the CPU-oracle sample (0: sized for roughly 15 s from a short probe)")
     ap.add_argument("--shape", default=None,
                     help="T,H,F,n,K,F_sh: a reduced layer with the recipe of --config (for profiler captures)")
-    ap.add_argument("--profile", action="store_true",
-                    help="only run warm-up + steps of the device-resident hot path, print a short line and exit")
+    ap.add_argument("--profile", nargs="?", const="step", default=None, choices=["step", "stages"],
+                    help="for profiler captures: only run warm-up + steps of the device-resident hot path (\"step\", the "
+                         "single call) or of the path taken stage by stage through the separate entry points "
+                         "(\"stages\"), print a short line and exit")
     ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
@@ -614,6 +668,9 @@ def main():
                     help="replay the hot path from a CUDA graph in the device-resident timing loop")
     ap.add_argument("--ffn-impl", type=int, default=0,
                     help="pcomoe_ffn_impl: 0 auto, 1 SIMT, 2 tcgen05 one CTA per tile, 3 tcgen05 CTA pairs")
+    ap.add_argument("--tp", action="store_true",
+                    help="with --gpus N: F-sliced tensor parallelism over the N ranks (one batch, strong scaling) "
+                         "instead of token data parallelism over replicas")
     ap.add_argument("--variant", default="default", choices=["default", "vanilla"],
                     help="vanilla: diagonal-only mask (every path a whole expert, no reuse)")
     args = ap.parse_args()
@@ -647,6 +704,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.tp:
+        run_tp(args, cfg, dev, rank, world, stream, barrier)
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     # Every rank holds a replica of the weights and its own batch of T tokens (token data parallel,
     # no collective on the data path); rank r draws its tokens with seed + 100*r.
     res = measure_config(args, cfg, args.config, dev, rank, world, stream, barrier, headline=True)
