@@ -325,8 +325,9 @@ pcomoe_status pcomoe_router_logits(const pcomoe_layer *layer, int32_t T, const v
  * block's input, as in any transformer block; the paper does not write this step out): 
  *     d_h_out[t,k] = round(d_h_in[t,k] + d_y[t,k])
  * one fp32 addition per element, rounded to nearest-even into the layer's storage type (exact copy of the sum
- * for fp32 layers).  d_h_in, d_h_out [T,H] in_dtype (may be the same array); d_y [T,H] fp32.  Asynchronous on
- * `stream`; allocates nothing.  Errors: INVALID_ARG, SHAPE (T < 0), CUDA. */
+ * for fp32 layers).  d_h_in, d_h_out [T,H] in_dtype (may be the same array); d_y [T,H] fp32 (a layer whose
+ * out_dtype is bf16 is refused with UNSUPPORTED).  Asynchronous on `stream`; allocates nothing.
+ * Errors: INVALID_ARG, SHAPE (T < 0), UNSUPPORTED, CUDA. */
 pcomoe_status pcomoe_residual_cast(const pcomoe_layer *layer, int32_t T, const void *d_h_in, const float *d_y,
                                    void *d_h_out, void *stream);
 

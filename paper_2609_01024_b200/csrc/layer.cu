@@ -379,6 +379,7 @@ pcomoe_status pcomoe_residual_cast(const pcomoe_layer *L, int32_t T, const void 
   if (T < 0) return PCOMOE_ERR_SHAPE;
   if (T == 0) return PCOMOE_OK;
   if (!d_h_in || !d_y || !d_h_out) return PCOMOE_ERR_INVALID_ARG;
+  if (L->cfg.out_dtype != PCOMOE_FP32) return PCOMOE_ERR_UNSUPPORTED;   // d_y is read as fp32
   return launch_residual_cast(L, T, d_h_in, d_y, d_h_out, (cudaStream_t)stream);
 }
 
