@@ -73,3 +73,39 @@ def test_host_side_argument_checks(lib):
     assert lib.pcomoe_mask_tighten(4, bias, m2, ctypes.c_float(0.5), m2) == 0                    # in place
     assert sum(m2) == 4 + 6
     assert lib.pcomoe_device_status(None, None) == 3
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own (no C++-isms), and a C caller must be
+    able to fill the structs and link against the library."""
+    import subprocess
+    hdr = os.path.join(ROOT, "include", "pcomoe.h")
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-fsyntax-only", "-x", "c", hdr], check=True)
+    src = tmp_path / "caller.c"
+    src.write_text("""
+#include <stdio.h>
+#include "pcomoe.h"
+int main(void) {
+  pcomoe_config cfg = {0};
+  pcomoe_layer *layer = 0;
+  unsigned char mask[4] = {1, 0, 0, 1};
+  float bias[4] = {0.f, 0.f, 0.f, 0.f};
+  cfg.struct_size = (int)sizeof cfg; cfg.n_experts = 2; cfg.top_k = 3; cfg.hidden = 64; cfg.ffn = 64;
+  cfg.in_dtype = PCOMOE_FP32; cfg.out_dtype = PCOMOE_FP32; cfg.norm_topk = 1; cfg.routed_scale = 1.0f; cfg.dedup = 1;
+  /* K > n: refused on the host, before any device is touched */
+  if (pcomoe_layer_create(&cfg, mask, bias, &layer) != PCOMOE_ERR_SHAPE) return 1;
+  if (pcomoe_set_wait_limit_us(61000000u) != PCOMOE_ERR_INVALID_ARG) return 2;
+  if (pcomoe_host_pipe_submit(0, 1, 0, 0, 0, 0) != PCOMOE_ERR_INVALID_ARG) return 3;
+  puts(pcomoe_status_string(PCOMOE_ERR_TIMEOUT));
+  return 0;
+}
+""")
+    from paper_2609_01024_b200 import build
+    lib = build.build()
+    exe = tmp_path / "caller"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe),
+                    lib, "-Wl,-rpath," + os.path.dirname(lib), "-L/usr/local/cuda/lib64", "-lcudart",
+                    "-Wl,-rpath,/usr/local/cuda/lib64", "-lstdc++"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stderr)
+    assert out.stdout.strip() == "device wait timed out"
