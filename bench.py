@@ -731,12 +731,14 @@ def main():
         per = {}
         for ci in (3, 4, 5):
             r = measure_config(args, wl.CONFIGS[ci], ci, dev, rank, world, stream, barrier, headline=False)
-            per[str(ci)] = {"workload": r["config"]["workload"], "T": wl.CONFIGS[ci].T, "ms_per_step": r["ms_per_step"],
+            cc = wl.CONFIGS[ci]
+            per[str(ci)] = {"workload": r["config"]["workload"], "T": cc.T, "H": cc.H, "F": cc.F, "n": cc.n, "K": cc.K,
+                            "F_sh": cc.F_sh, "ms_per_step": r["ms_per_step"],
                             "tokens_per_s": r["value"], "R1_over_P": r["config"]["R1_over_P"],
                             "e2e_tokens_per_s": r["e2e"]["value"], "e2e_bf16_y_tokens_per_s": r["e2e_bf16_y"]["value"],
                             "gpu_launches": r["launches"], "stage_ms": r["stage_ms"],
-                            "roofline": {k: r["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "traffic")},
-                            "roofline_sustained": {k: r["roofline_sustained"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "ms_per_step")},
+                            "roofline": {k: r["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "traffic", "algorithmic", "kernel")},
+                            "roofline_sustained": {k: r["roofline_sustained"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "ms_per_step", "stage_ms")},
                             "layer_frac_burst": r["layer_roofline"]["frac_burst"],
                             "layer_frac_sustained": r["layer_roofline"]["frac_sustained"],
                             "layer_frac_of_nominal_2.25PF_8TBs": r["layer_roofline"]["frac_of_nominal_2.25PF_8TBs"],
