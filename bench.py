@@ -402,13 +402,14 @@ def dominant_roofline(cfg, work, n_src, stage_ms, peak_tflops, peak_gbs, regime,
         return {"bound": "tensor", "achieved": ach, "peak": peak_tflops, "unit": "TFLOP/s", "frac": ach / peak_tflops,
                 "traffic": traffic, "regime": regime, "timed_region": region,
                 "kernel": "stage-1 grouped GEMM over the routed groups (row gather + grouped_gemm_pair_kernel<1>)",
-                "algorithmic": "4*R1*H*F FLOP per launch", "peak_source": source}
+                "algorithmic": "4*R1*H*F FLOP per launch", "algorithmic_value": work["flops_s1"], "peak_source": source}
     s1_bytes = (2 if tc_path else 4) * (2 * n_src * cfg.H * cfg.F)
     ach = s1_bytes / t / 1e9
     return {"bound": "hbm", "achieved": ach, "peak": peak_gbs, "unit": "GB/s", "frac": ach / peak_gbs,
             "traffic": traffic, "regime": regime, "timed_region": region,
             "kernel": "stage-1 grouped GEMM, routed groups (weight streaming, grouped_gemm_kernel<1>)",
-            "algorithmic": "2*n_src*H*F*sizeof(weight) bytes per launch", "peak_source": source}
+            "algorithmic": "2*n_src*H*F*sizeof(weight) bytes per launch", "algorithmic_value": s1_bytes,
+            "peak_source": source}
 
 
 def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, headline):
@@ -737,7 +738,7 @@ def main():
                             "tokens_per_s": r["value"], "R1_over_P": r["config"]["R1_over_P"],
                             "e2e_tokens_per_s": r["e2e"]["value"], "e2e_bf16_y_tokens_per_s": r["e2e_bf16_y"]["value"],
                             "gpu_launches": r["launches"], "stage_ms": r["stage_ms"],
-                            "roofline": {k: r["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "traffic", "algorithmic", "kernel")},
+                            "roofline": {k: r["roofline"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "traffic", "algorithmic", "algorithmic_value", "kernel")},
                             "roofline_sustained": {k: r["roofline_sustained"][k] for k in ("bound", "achieved", "peak", "unit", "frac", "regime", "ms_per_step", "stage_ms")},
                             "layer_frac_burst": r["layer_roofline"]["frac_burst"],
                             "layer_frac_sustained": r["layer_roofline"]["frac_sustained"],
