@@ -420,6 +420,8 @@ def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, h
     local = int(os.environ.get("LOCAL_RANK", "0"))
     L = wl.make_layer(cfg)                              # same mask, bias and weights on every rank
     L.h, L.logits = replicas.rank_inputs(cfg, rank)     # its own batch of tokens
+    if args.variant == "half_c":
+        L.bias = wl.make_bias(cfg, c_scale=0.5)
     layer = build_layer(args, cfg, L, dev)
     d_logits = torch.from_numpy(L.logits).to(dev)
     d_h = B.to_device(L.h, dev)
@@ -672,8 +674,10 @@ def main():
     ap.add_argument("--tp", action="store_true",
                     help="with --gpus N: F-sliced tensor parallelism over the N ranks (one batch, strong scaling) "
                          "instead of token data parallelism over replicas")
-    ap.add_argument("--variant", default="default", choices=["default", "vanilla"],
-                    help="vanilla: diagonal-only mask (every path a whole expert, no reuse)")
+    ap.add_argument("--variant", default="default", choices=["default", "vanilla", "half_c"],
+                    help="vanilla: diagonal-only mask (every path a whole expert, no reuse); half_c: the off-diagonal "
+                         "prior of the compatibility bias halved (c = -sigma_z/2), so that more off-diagonal paths are "
+                         "chosen and more stage-1 rows are shared")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = wl.CONFIGS[args.config]
