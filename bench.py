@@ -735,7 +735,11 @@ def main():
     if res is not None and world == 1 and plain and not args.no_per_config:
         per = {}
         for ci in (3, 4, 5):
-            r = measure_config(args, wl.CONFIGS[ci], ci, dev, rank, world, stream, barrier, headline=False)
+            try:
+                r = measure_config(args, wl.CONFIGS[ci], ci, dev, rank, world, stream, barrier, headline=False)
+            except Exception as e:   # the headline line is printed whatever happens to an extra configuration
+                per[str(ci)] = {"workload": wl.CONFIGS[ci].name, "error": f"{type(e).__name__}: {e}"}
+                continue
             cc = wl.CONFIGS[ci]
             per[str(ci)] = {"workload": r["config"]["workload"], "T": cc.T, "H": cc.H, "F": cc.F, "n": cc.n, "K": cc.K,
                             "F_sh": cc.F_sh, "ms_per_step": r["ms_per_step"],
