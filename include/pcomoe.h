@@ -246,7 +246,8 @@ pcomoe_status pcomoe_ffn_forward(const pcomoe_layer *layer, int32_t T, const voi
 /* The pieces of pcomoe_ffn_forward one by one, for timing and for checking a stage alone (same
  * arguments and errors).  `stages` is a bit mask: 1 = stage 1 over the routed groups, 2 = stage 1 of
  * the shared expert, 4 = zero-fill of y and stage 2 over the routed groups, 8 = stage 2 of the shared
- * expert.  pcomoe_ffn_forward is stages = 15.  Stage 2 reads what stage 1 left in the workspace. */
+ * expert.  pcomoe_ffn_forward is stages = 15.  Stage 2 reads what stage 1 left in the workspace.  With a bf16
+ * output the rounded y is rewritten from the fp32 sum after every call that includes bit 4 or bit 8. */
 pcomoe_status pcomoe_ffn_forward_stages(const pcomoe_layer *layer, int32_t T, const void *d_h,
                                         const void *d_w_gate, const void *d_w_up,
                                         const void *d_w_down, const void *d_wsh_gate,
