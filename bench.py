@@ -446,6 +446,24 @@ def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, h
     for _ in range(args.warmup):
         step()
     assert layer.device_status() == 0, "device reported an error during warm-up"
+    if headline and args.timeline:
+        # start and end of every kernel of one step of the single call, streams overlapped as they run live
+        # (CUPTI activity records through torch.profiler; a kernel launched early by programmatic dependent launch
+        # "starts" when it becomes resident and then waits, so read the END times)
+        from torch.profiler import ProfilerActivity, profile
+        with profile(activities=[ProfilerActivity.CUDA]) as prof:
+            for _ in range(4):
+                step()
+            torch.cuda.synchronize()
+        ev = sorted((e for e in prof.events() if e.device_type == torch.autograd.DeviceType.CUDA),
+                    key=lambda e: e.time_range.start)
+        per = len(ev) // 4
+        t0 = ev[2 * per].time_range.start
+        rows = [{"start_us": round(e.time_range.start - t0, 1), "end_us": round(e.time_range.end - t0, 1),
+                 "kernel": e.name.replace("(anonymous namespace)::", "").replace("pcomoe::", "").split("(")[0][:70]}
+                for e in ev[2 * per: 3 * per]]
+        print(json.dumps({"timeline_of": cfg.name, "third_of_four_steps": rows}))
+        return None
     if headline and args.profile:
         if args.profile == "stages":
             time_stages(layer, cfg, d_logits, d_h, stream, with_router, args.steps, 0)
@@ -652,6 +670,8 @@ def main():
                     help="for profiler captures: only run warm-up + steps of the device-resident hot path (\"step\", the "
                          "single call) or of the path taken stage by stage through the separate entry points "
                          "(\"stages\"), print a short line and exit")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print start and end of every kernel of one step of the single call (streams overlapped as live) and exit")
     ap.add_argument("--ref-tokens", type=int, default=32, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
@@ -731,7 +751,7 @@ def main():
     # The other benchmark layers, timed the same way after the headline (one GPU only: the scaling runs repeat the
     # headline configuration at every N).
     plain = (args.config == 2 and not args.shape and args.variant == "default" and args.router < 0 and not args.graph
-             and args.layers == 0 and not args.profile and args.target_reuse == 0 and args.ffn_impl == 0)
+             and args.layers == 0 and not args.profile and not args.timeline and args.target_reuse == 0 and args.ffn_impl == 0)
     if res is not None and world == 1 and plain and not args.no_per_config:
         per = {}
         for ci in (3, 4, 5):
