@@ -1,6 +1,9 @@
-// Glue between the layers of a decode-step loop: the residual stream.  h_out = round_to_storage(h_in + y), where y
-// is a layer's fp32 output and h the hidden states in the layers' storage type.  The add is one fp32 operation and
-// the rounding to bf16 is round-to-nearest-even, so the next layer's input is a defined bit pattern.
+// Small kernels around the layer.
+//   residual stream between the layers of a decode-step loop: h_out = round_to_storage(h_in + y), where y is a
+//     layer's fp32 output and h the hidden states in the layers' storage type; the add is one fp32 operation and the
+//     rounding to bf16 is round-to-nearest-even, so the next layer's input is a defined bit pattern;
+//   bf16 output type: the fp32 sum of the layer rounded once, after the last addition;
+//   self-test of the bounded device-side wait (failure detection without hanging anything).
 #include <algorithm>
 #include <cuda_bf16.h>
 
