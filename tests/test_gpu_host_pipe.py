@@ -95,3 +95,16 @@ def test_bf16_output_small_shapes(G, oracle, impl):
         G.check_output(y.float().cpu().numpy(), _reference(oracle, c, L, L.h[:T], L.logits[:T]))
         y3 = layer.forward_three_calls(dl[:T], dh[:T]).float().cpu().numpy()
         G.check_output(y3, _reference(oracle, c, L, L.h[:T], L.logits[:T]))
+
+
+def test_residual_hand_over_refuses_a_bf16_output_layer(G):
+    """pcomoe_residual_cast reads y as fp32: a layer whose output type is bf16 is refused, not misread."""
+    cfg = wl.small_case(58, T=64, H=256, F=128, n=4, K=2)
+    L = wl.make_layer(cfg)
+    layer = G.make_gpu_layer(cfg, L, out_dtype=G.B.PCOMOE_BF16)
+    h = G.B.to_device(L.h)
+    y = layer.forward(torch.from_numpy(L.logits).to(layer.device), h)
+    out = torch.empty_like(h)
+    with pytest.raises(G.B.PcomoeError) as e:
+        G.B.pcomoe_residual_cast(layer.layer, cfg.T, h, y, out)
+    assert e.value.status == 4          # PCOMOE_ERR_UNSUPPORTED
