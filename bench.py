@@ -484,13 +484,16 @@ def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, h
     barrier()
     n0 = B.pcomoe_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]   # one more event per step: median / min
     t_wall0 = time.time()
     e0.record(stream)
-    for _ in range(args.steps):
+    for i in range(args.steps):
         step()
+        step_marks[i].record(stream)
     e1.record(stream)
     barrier()
     t_wall1 = time.time()
+    per_step = [(e0 if i == 0 else step_marks[i - 1]).elapsed_time(step_marks[i]) for i in range(args.steps)]
     launches = B.pcomoe_launch_count() - n0
     if headline and args.graph:   # replays do not pass through the library's launch counter: count the captured launches
         m0 = B.pcomoe_launch_count(); layer.forward(d_logits, d_h); launches = (B.pcomoe_launch_count() - m0) * args.steps
@@ -577,7 +580,8 @@ def measure_config(args, cfg, config_index, dev, rank, world, stream, barrier, h
                       "note": "frac_burst: the headline loop's ms_per_step (tens of ms from warm clocks) over the burst "
                               "peaks; frac_sustained: ms_per_step after 1 s of continuous steps over the sustained peak"}
     tc_path = cfg.dtype == "bf16"
-    res = {"ms_per_step": ms_per_step, "value": value, "e2e": e2e, "e2e_bf16_y": e2e_bf16, "launches": int(launches),
+    res = {"ms_per_step": ms_per_step, "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
+           "value": value, "e2e": e2e, "e2e_bf16_y": e2e_bf16, "launches": int(launches),
            "clocks": clocks, "roofline": roofline, "roofline_sustained": roofline_sus, "layer_roofline": layer_roofline,
            "stage_ms": burst_mean, "dtype": "bf16" if tc_path else "f32",
            "config": {"workload": cfg.name, "variant": args.variant, "T": cfg.T, "H": cfg.H, "F": cfg.F,
@@ -740,7 +744,8 @@ def main():
     res = measure_config(args, cfg, args.config, dev, rank, world, stream, barrier, headline=True)
     if res is not None and rank == 0:
         out = {"metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
-               "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+               "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "ms_per_step_median": res["ms_per_step_median"],
+               "ms_per_step_min": res["ms_per_step_min"], "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": res["dtype"], "data": "synthetic", "config": res["config"],
                "e2e": res["e2e"], "e2e_bf16_y": res["e2e_bf16_y"], "gpu_launches": res["launches"],
                "clocks": res["clocks"], "roofline": res["roofline"], "roofline_sustained": res["roofline_sustained"],
